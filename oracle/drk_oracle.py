@@ -1,0 +1,306 @@
+"""fp64 CPU oracle for the fused policy-gradient loss over the LM head.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain definition that the
+CUDA library is checked against.  Only the test-suite, the smoke check and the
+CPU-baseline leg of the benchmark may import it; the product path never does.
+It shares no code with the CUDA sources and never receives values produced by
+them (the one exception is the documented `keep_override`, used by the parity
+comparator for segments whose accept/reject decision lies inside rounding
+distance of a threshold).
+
+Everything is numpy float64.  `np.matmul` serves as the library primitive for
+the three dense contractions; there is no blocking, fusion or reordering.
+
+What follows the paper, and where:
+
+  returns()            reward-to-go return                      Sec. 4.2, Eq. 2
+  grpo_advantage()     turn-group mean baseline                 Sec. 4.2, Eq. 3
+  trloo_advantage()    leave-one-out turn-level advantage       Sec. 4.2, Eq. 5
+  mrs()                geometric mismatch rejection sampling    Sec. 5.1 (unnumbered eq.)
+                       with the token-level veto
+  coeff_and_loss()     REINFORCE surrogate                      App. A (estimator g-hat)
+  logits()/token_logprob()/gradients()
+                       the plain definition of log-softmax over the LM head
+                       and its analytic gradient (the paper names the trainer
+                       log-probability pi_train(a_t|s_t) but not how it is
+                       computed; the definition is the textbook one).
+
+Parity pins: every function here is pinned by tests that run without a GPU
+(closed forms, brute force, finite differences, a float64 library
+cross-check and the worked three-turn example of App. E); none is unpinned.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass
+
+import numpy as np
+
+F64 = np.float64
+
+# Constants printed in Sec. 5.1.
+MRS_LO = 0.999
+MRS_HI = 1.001
+MRS_VETO = 1e-4
+
+NORM_KEPT_TOKENS = 0
+NORM_ALL_MASKED_TOKENS = 1
+NORM_EXPLICIT = 2
+
+
+# ---------------------------------------------------------------------------
+# Returns and advantages (Sec. 4.2)
+# ---------------------------------------------------------------------------
+
+def returns(reward, valid, gamma=1.0):
+    """Eq. 2: G[i,t] = sum_{t'>=t} gamma^(t'-t) R[i,t'].
+
+    A rollout that ended early has no reward at its later turns: only valid
+    turns t' contribute, and an invalid (i,t) has G = 0.
+    """
+    reward = np.asarray(reward, dtype=F64)
+    valid = np.asarray(valid).astype(bool)
+    R, Tmax = reward.shape
+    G = np.zeros((R, Tmax), dtype=F64)
+    for i in range(R):
+        for t in range(Tmax):
+            if not valid[i, t]:
+                continue
+            acc = 0.0
+            for tp in range(t, Tmax):
+                if valid[i, tp]:
+                    acc += (float(gamma) ** (tp - t)) * reward[i, tp]
+            G[i, t] = acc
+    return G
+
+
+def turn_groups(valid, prompt_of_rollout):
+    """The sets G_t of Sec. 4.2: for every prompt p and turn t, the valid
+    rollouts of p at t.  Returns a list of (t, [rollout indices])."""
+    valid = np.asarray(valid).astype(bool)
+    prompt_of_rollout = np.asarray(prompt_of_rollout)
+    R, Tmax = valid.shape
+    groups = []
+    for p in np.unique(prompt_of_rollout):
+        members = [i for i in range(R) if prompt_of_rollout[i] == p]
+        for t in range(Tmax):
+            g = [i for i in members if valid[i, t]]
+            if g:
+                groups.append((t, g))
+    return groups
+
+
+def grpo_advantage(G, valid, prompt_of_rollout):
+    """Eq. 3: A[i,t] = G[i,t] - mean_{j in G_t} G[j,t].  Returns (A, N)."""
+    G = np.asarray(G, dtype=F64)
+    A = np.zeros_like(G)
+    N = np.zeros(G.shape, dtype=np.int64)
+    for t, g in turn_groups(valid, prompt_of_rollout):
+        n = len(g)
+        mean = sum(G[j, t] for j in g) / n
+        for i in g:
+            A[i, t] = G[i, t] - mean
+            N[i, t] = n
+    return A, N
+
+
+def trloo_advantage(G, valid, prompt_of_rollout):
+    """Eq. 5: A[i,t] = G[i,t] - (1/(N_t-1)) sum_{j in G_t, j != i} G[j,t].
+
+    The paper defines it for N_t > 1 only; a group of one has no other
+    rollout to form a baseline from and gets advantage 0, as does every
+    invalid (i,t).  Returns (A, N) with N[i,t] = N_t (0 where invalid).
+    """
+    G = np.asarray(G, dtype=F64)
+    A = np.zeros_like(G)
+    N = np.zeros(G.shape, dtype=np.int64)
+    for t, g in turn_groups(valid, prompt_of_rollout):
+        n = len(g)
+        for i in g:
+            N[i, t] = n
+            if n > 1:
+                others = sum(G[j, t] for j in g if j != i)
+                A[i, t] = G[i, t] - others / (n - 1)
+    return A, N
+
+
+# ---------------------------------------------------------------------------
+# LM head: logits, log-softmax, gather
+# ---------------------------------------------------------------------------
+
+def logits(hidden, W):
+    """s[t,v] = sum_h hidden[t,h] * W[v,h] (all of them)."""
+    return np.matmul(np.asarray(hidden, dtype=F64), np.asarray(W, dtype=F64).T)
+
+
+def logsumexp_rows(s):
+    """lse[t] = max_v s[t,v] + ln sum_v exp(s[t,v] - max_v s[t,v])."""
+    m = np.max(s, axis=1)
+    return m + np.log(np.sum(np.exp(s - m[:, None]), axis=1))
+
+
+def token_logprob(s, ids):
+    """log pi(ids[t] | row t) = s[t, ids[t]] - lse[t].  Returns (logp, lse)."""
+    ids = np.asarray(ids, dtype=np.int64)
+    lse = logsumexp_rows(s)
+    tgt = s[np.arange(s.shape[0]), ids]
+    return tgt - lse, lse
+
+
+# ---------------------------------------------------------------------------
+# Mismatch rejection sampling (Sec. 5.1)
+# ---------------------------------------------------------------------------
+
+@dataclass
+class MrsResult:
+    w: np.ndarray           # [S] geometric-mean importance ratio
+    keep: np.ndarray        # [S] bool
+    vetoed: np.ndarray      # [S] bool, token veto fired
+    mean_delta: np.ndarray  # [S] mean log ratio over the segment's masked tokens
+    min_delta: np.ndarray   # [S] smallest token log ratio (+inf for empty segments)
+    n_masked: np.ndarray    # [S] int64
+    margin: np.ndarray      # [S] distance (log space) of the decision to the nearest threshold
+
+
+def mrs(logp, rollout_logp, loss_mask, cu_seqlens, lo=MRS_LO, hi=MRS_HI, veto=MRS_VETO):
+    """Geometric MRS with token veto, one decision per training sample.
+
+    For the masked tokens M of a segment: delta_t = logp_t - rollout_logp_t,
+    w = exp(mean_M delta).  The sample is retained iff lo <= w <= hi and no
+    token's ratio exp(delta_t) is below `veto`.  Both tests are taken in log
+    space (ln lo <= mean delta <= ln hi; min delta >= ln veto).  lo <= 0
+    removes the lower bound, hi = inf the upper one, veto <= 0 the veto.
+    A segment without masked tokens has w = 1 and is not retained.
+    """
+    logp = np.asarray(logp, dtype=F64)
+    rollout_logp = np.asarray(rollout_logp, dtype=F64)
+    loss_mask = np.asarray(loss_mask).astype(bool)
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    S = cu.shape[0] - 1
+    ln_lo = math.log(lo) if lo > 0 else -math.inf
+    ln_hi = math.log(hi) if math.isfinite(hi) else math.inf
+    ln_veto = math.log(veto) if veto > 0 else -math.inf
+    w = np.ones(S, dtype=F64)
+    keep = np.zeros(S, dtype=bool)
+    vetoed = np.zeros(S, dtype=bool)
+    mean_delta = np.zeros(S, dtype=F64)
+    min_delta = np.full(S, np.inf, dtype=F64)
+    n_masked = np.zeros(S, dtype=np.int64)
+    margin = np.full(S, np.inf, dtype=F64)
+    for g in range(S):
+        a, b = int(cu[g]), int(cu[g + 1])
+        m = loss_mask[a:b]
+        n = int(m.sum())
+        n_masked[g] = n
+        if n == 0:
+            continue
+        delta = (logp[a:b] - rollout_logp[a:b])[m]
+        mean_delta[g] = delta.sum() / n
+        min_delta[g] = delta.min()
+        w[g] = math.exp(mean_delta[g])
+        in_band = (ln_lo <= mean_delta[g]) and (mean_delta[g] <= ln_hi)
+        vetoed[g] = min_delta[g] < ln_veto
+        keep[g] = in_band and not vetoed[g]
+        margin[g] = min(abs(mean_delta[g] - ln_lo), abs(mean_delta[g] - ln_hi),
+                        abs(min_delta[g] - ln_veto))
+    return MrsResult(w, keep, vetoed, mean_delta, min_delta, n_masked, margin)
+
+
+# ---------------------------------------------------------------------------
+# Coefficients and the loss (App. A)
+# ---------------------------------------------------------------------------
+
+@dataclass
+class LossResult:
+    coeff: np.ndarray     # [T] coefficient c_t that multiplies grad log pi at token t
+    loss: float
+    scale: float
+    kept_tokens: int
+    masked_tokens: int
+    kept_segs: int
+
+
+def coeff_and_loss(logp, keep, loss_mask, cu_seqlens, seg_adv,
+                   norm=NORM_KEPT_TOKENS, explicit_scale=1.0):
+    """c_t = keep_seg(t) * mask_t * A_seg(t) * scale, loss = -sum_t c_t logp_t.
+
+    The estimator of App. A sums grad log pi(y_{i,t}|s_{i,t}) * A_{i,t} over
+    samples; log pi of a response is the sum of its token log-probs, so every
+    masked token of a retained sample carries the sample's advantage.  The
+    outer averaging convention is left open by the paper: `norm` picks
+    1/(kept masked tokens), 1/(all masked tokens) or a caller constant.
+    Tokens outside [cu[0], cu[S]) belong to no sample and get c_t = 0.
+    """
+    logp = np.asarray(logp, dtype=F64)
+    loss_mask = np.asarray(loss_mask).astype(bool)
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    keep = np.asarray(keep).astype(bool)
+    seg_adv = np.asarray(seg_adv, dtype=F64)
+    S = cu.shape[0] - 1
+    T = logp.shape[0]
+    kept_tokens = 0
+    masked_tokens = 0
+    for g in range(S):
+        n = int(loss_mask[cu[g]:cu[g + 1]].sum())
+        masked_tokens += n
+        if keep[g]:
+            kept_tokens += n
+    if norm == NORM_KEPT_TOKENS:
+        scale = 1.0 / max(kept_tokens, 1)
+    elif norm == NORM_ALL_MASKED_TOKENS:
+        scale = 1.0 / max(masked_tokens, 1)
+    elif norm == NORM_EXPLICIT:
+        scale = float(explicit_scale)
+    else:
+        raise ValueError("unknown norm")
+    coeff = np.zeros(T, dtype=F64)
+    for g in range(S):
+        if not keep[g]:
+            continue
+        a, b = int(cu[g]), int(cu[g + 1])
+        coeff[a:b] = np.where(loss_mask[a:b], seg_adv[g] * scale, 0.0)
+    loss = -float(np.sum(coeff * logp))
+    return LossResult(coeff, loss, scale, kept_tokens, masked_tokens, int(keep.sum()))
+
+
+# ---------------------------------------------------------------------------
+# Gradients of the loss w.r.t. hidden and W (c_t held constant)
+# ---------------------------------------------------------------------------
+
+def dlogits(s, lse, ids, coeff):
+    """dL[t,v] = c_t * (softmax(s)[t,v] - [v == ids[t]])."""
+    p = np.exp(s - np.asarray(lse, dtype=F64)[:, None])
+    p[np.arange(s.shape[0]), np.asarray(ids, dtype=np.int64)] -= 1.0
+    return p * np.asarray(coeff, dtype=F64)[:, None]
+
+
+def gradients(hidden, W, s, lse, ids, coeff):
+    """dH[t,:] = sum_v dL[t,v] W[v,:];  dW[v,:] = sum_t dL[t,v] hidden[t,:]."""
+    dL = dlogits(s, lse, ids, coeff)
+    dH = np.matmul(dL, np.asarray(W, dtype=F64))
+    dW = np.matmul(dL.T, np.asarray(hidden, dtype=F64))
+    return dH, dW
+
+
+# ---------------------------------------------------------------------------
+# The whole path for one packed micro-batch
+# ---------------------------------------------------------------------------
+
+def pg_loss_fwd_bwd(hidden, W, ids, rollout_logp, loss_mask, cu_seqlens, seg_adv,
+                    lo=MRS_LO, hi=MRS_HI, veto=MRS_VETO,
+                    norm=NORM_KEPT_TOKENS, explicit_scale=1.0,
+                    keep_override=None, want_grads=True):
+    """Forward, MRS, loss and (optionally) gradients.  Returns a dict."""
+    s = logits(hidden, W)
+    logp, lse = token_logprob(s, ids)
+    m = mrs(logp, rollout_logp, loss_mask, cu_seqlens, lo, hi, veto)
+    keep = m.keep if keep_override is None else np.asarray(keep_override).astype(bool)
+    lr = coeff_and_loss(logp, keep, loss_mask, cu_seqlens, seg_adv, norm, explicit_scale)
+    out = dict(logp=logp, lse=lse, mrs=m, keep=keep, coeff=lr.coeff, loss=lr.loss,
+               scale=lr.scale, kept_tokens=lr.kept_tokens, masked_tokens=lr.masked_tokens,
+               kept_segs=lr.kept_segs, vetoed_segs=int(m.vetoed.sum()))
+    if want_grads:
+        dH, dW = gradients(hidden, W, s, lse, ids, lr.coeff)
+        out["dH"] = dH
+        out["dW"] = dW
+    return out
