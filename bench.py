@@ -1,0 +1,340 @@
+#!/usr/bin/env python
+"""Throughput of the fused policy-gradient loss (TRLOO + MRS + LM-head fwd/bwd) on synthetic batches.
+
+    python bench.py --gpus 1 --steps 10 --warmup 3
+    python -m torch.distributed.run --nnodes=1 --nproc-per-node N ... bench.py --gpus N ...
+    python bench.py --impl reference ...     # times the fp64 CPU oracle on a bounded sample
+
+One step = one pass of the whole path over one packed micro-batch: drk_trloo_advantage over the rollout
+batch, the caller's gather of per-sample advantages, drk_pg_loss_fwd_bwd.  Prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "fused PG-loss fwd+bwd tokens/s at H=5120,V=151936 bf16; % of dense BF16 peak"
+UNIT = "tokens/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(tflops=float(d["bf16_tflops_sustained"]), burst=float(d["bf16_tflops"]),
+                    hbm=float(d["hbm_gbs"]), source="measured")
+    return dict(tflops=1400.0, burst=1590.0, hbm=6650.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    samples=len(sm), reasons=sorted(reasons))
+
+
+def run_reference(args):
+    """Times the oracle, as it stands, on the host cores: each step is a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    from oracle import drk_oracle as O
+    from paper_2602_05885_b200 import workload
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    n_tok = args.ref_tokens
+    wl = workload.build("qwen3-14b", "cpu", seed=2000, T_override=n_tok)
+    hidden = wl.hidden.double().numpy()
+    W = wl.W.double().numpy()
+    ids = wl.ids.numpy()
+    rl = wl.rollout_logp.double().numpy()
+    mask = wl.loss_mask.numpy()
+    cu = wl.cu.numpy()
+    adv = np.ones(wl.S)
+    lo, hi = wl.wide_band()
+
+    def step():
+        G = O.returns(wl.reward.numpy(), wl.valid.numpy(), 1.0)
+        O.trloo_advantage(G, wl.valid.numpy(), wl.prompt_of_rollout.numpy())
+        return O.pg_loss_fwd_bwd(hidden, W, ids, rl, mask, cu, adv, lo=lo, hi=hi)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    val = n_tok * args.steps / dt
+    sample = f"{n_tok} packed tokens per step at full H=5120, V=151936 (fp64 oracle: TRLOO + fwd + MRS + loss + dH + dW)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "qwen3-14b-shaped micro-batch, H=5120, V=151936", "sample_tokens": n_tok},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def cpu_baseline(n_tok: int):
+    """The oracle timed once on a bounded sample of the same workload (host cores of this machine)."""
+    import numpy as np
+    from oracle import drk_oracle as O
+    from paper_2602_05885_b200 import workload
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    wl = workload.build("qwen3-14b", "cpu", seed=2000, T_override=n_tok)
+    hidden = wl.hidden.double().numpy()
+    W = wl.W.double().numpy()
+    lo, hi = wl.wide_band()
+    t0 = time.perf_counter()
+    G = O.returns(wl.reward.numpy(), wl.valid.numpy(), 1.0)
+    O.trloo_advantage(G, wl.valid.numpy(), wl.prompt_of_rollout.numpy())
+    O.pg_loss_fwd_bwd(hidden, W, wl.ids.numpy(), wl.rollout_logp.double().numpy(), wl.loss_mask.numpy(),
+                      wl.cu.numpy(), np.ones(wl.S), lo=lo, hi=hi)
+    dt = time.perf_counter() - t0
+    return {"value": n_tok / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"one pass over {n_tok} packed tokens at full H=5120, V=151936 in {dt:.1f} s "
+                      "(fp64: TRLOO + full logits + log-softmax + MRS + loss + dH + dW)"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="qwen3-14b", choices=["qwen3-14b", "qwen3-8b", "ragged", "tiny"])
+    ap.add_argument("--tokens", type=int, default=0, help="override the micro-batch size T (smaller captures)")
+    ap.add_argument("--dw-dtype", default="f32", choices=["f32", "bf16"])
+    ap.add_argument("--dh-dtype", default="bf16", choices=["f32", "bf16"])
+    ap.add_argument("--v-chunk", type=int, default=0)
+    ap.add_argument("--mrs", default="wide", choices=["wide", "paper", "off"])
+    ap.add_argument("--ref-tokens", type=int, default=256)
+    ap.add_argument("--cpu-tokens", type=int, default=512)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    from paper_2602_05885_b200 import binding as B
+    from paper_2602_05885_b200 import dp, workload
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    B.load()
+
+    # every rank owns a different micro-batch of the same rollout batch (weak scaling)
+    wl = workload.build(args.workload, dev, seed=2000, microbatch=rank, T_override=args.tokens or None)
+    T, H, V, S = wl.T, wl.H, wl.V, wl.S
+    code = B.DRK_F32 if wl.dtype == torch.float32 else B.DRK_BF16
+    p = B.drk_pg_params_default()
+    if args.mrs == "wide":
+        p.mrs_lo, p.mrs_hi = wl.wide_band()
+    elif args.mrs == "off":
+        p.mrs_lo, p.mrs_hi, p.veto_ratio = 0.0, float("inf"), 0.0
+    p.dw_dtype = B.DRK_BF16 if args.dw_dtype == "bf16" else B.DRK_F32
+    p.dh_dtype = B.DRK_BF16 if args.dh_dtype == "bf16" else B.DRK_F32
+    p.v_chunk = args.v_chunk
+    bufs = B.PgLossBuffers(T, H, V, S, code, p, dev)
+    R, Tmax = wl.reward.shape
+    ret = torch.empty_like(wl.reward)
+    adv = torch.empty_like(wl.reward)
+    gsize = torch.empty((R, Tmax), dtype=torch.int32, device=dev)
+    seg_flat = (wl.seg_rollout * Tmax + wl.seg_turn).contiguous()
+    stream = torch.cuda.current_stream()
+    launches = [0]
+
+    def step(hidden, ids, rl, mask, cu):
+        B.drk_trloo_advantage(wl.reward, wl.valid, wl.prompt_of_rollout, R, Tmax, 1.0, B.DRK_BASELINE_TRLOO,
+                              ret, adv, gsize, stream)
+        launches[0] += B.drk_last_launch_count()
+        seg_adv = adv.view(-1).index_select(0, seg_flat)     # the caller's gather of per-sample advantages
+        B.drk_pg_loss_fwd_bwd(hidden, wl.W, code, ids, rl, mask, cu, seg_adv, T, H, V, S, p, bufs.loss, bufs.logp,
+                              bufs.lse, bufs.seg_w, bufs.seg_keep, bufs.counters, bufs.dH, bufs.dW,
+                              bufs.workspace, bufs.workspace_bytes, bufs.status, stream)
+        launches[0] += B.drk_last_launch_count()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---------------------------------------------------------------- device-resident timing
+    for _ in range(args.warmup):
+        step(wl.hidden, wl.ids, wl.rollout_logp, wl.loss_mask, wl.cu)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches[0] = 0
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step(wl.hidden, wl.ids, wl.rollout_logp, wl.loss_mask, wl.cu)
+    ev1.record(stream)
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop() if rank == 0 else None
+    n_launch = launches[0]
+    status = int(bufs.status.item())
+    counters = bufs.counters.tolist()
+    ms_max = dp.max_over_ranks(ms, dev)
+    value = world * T * args.steps / (ms_max * 1e-3)
+
+    # ---------------------------------------------------------------- the fused call alone (roofline)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    seg_adv = adv.view(-1).index_select(0, seg_flat)
+    call_ms = []
+    for _ in range(min(args.steps, 5)):
+        e0.record(stream)
+        B.drk_pg_loss_fwd_bwd(wl.hidden, wl.W, code, wl.ids, wl.rollout_logp, wl.loss_mask, wl.cu, seg_adv, T, H, V, S,
+                              p, bufs.loss, bufs.logp, bufs.lse, bufs.seg_w, bufs.seg_keep, bufs.counters, bufs.dH,
+                              bufs.dW, bufs.workspace, bufs.workspace_bytes, bufs.status, stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        call_ms.append(e0.elapsed_time(e1))
+    n_gemm_launches = B.drk_last_launch_count() - 5     # all but merge + 3 MRS kernels + (bf16 dH: none extra)
+    fused_ms = statistics.mean(call_ms)
+    flops = 8.0 * T * H * V
+    peaks = measured_peaks()
+    achieved = flops / (fused_ms * 1e-3) / 1e12
+
+    # ---------------------------------------------------------------- end to end with host buffers
+    e2e = None
+    if not args.no_e2e:
+        host = [t.cpu().pin_memory() for t in (wl.hidden, wl.ids, wl.rollout_logp, wl.loss_mask, wl.cu)]
+        devin = [torch.empty_like(t, device=dev) for t in host]
+        h_loss = torch.empty(1, dtype=torch.float32).pin_memory()
+        h_cnt = torch.empty(4, dtype=torch.int64).pin_memory()
+        h_logp = torch.empty(T, dtype=torch.float32).pin_memory()
+        h_keep = torch.empty(S, dtype=torch.uint8).pin_memory()
+        h_dH = torch.empty((T, H), dtype=bufs.dH.dtype).pin_memory()
+        h2d = sum(t.numel() * t.element_size() for t in host)
+        d2h = sum(t.numel() * t.element_size() for t in (h_loss, h_cnt, h_logp, h_keep, h_dH))
+
+        def e2e_step():
+            for src, dst in zip(host, devin):
+                dst.copy_(src, non_blocking=True)
+            step(*devin)
+            h_loss.copy_(bufs.loss, non_blocking=True)
+            h_cnt.copy_(bufs.counters, non_blocking=True)
+            h_logp.copy_(bufs.logp, non_blocking=True)
+            h_keep.copy_(bufs.seg_keep, non_blocking=True)
+            h_dH.copy_(bufs.dH, non_blocking=True)
+
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        ev0.record(stream)
+        for _ in range(args.steps):
+            e2e_step()
+        ev1.record(stream)
+        barrier()
+        e_ms = dp.max_over_ranks(ev0.elapsed_time(ev1), dev)
+        e2e = {"value": world * T * args.steps / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e_ms / args.steps,
+               "what": "hidden, ids, rollout log-probs, mask, cu_seqlens copied from pinned host memory each step; "
+                       "loss, counters, log-probs, keep flags and dH copied back; W and dW stay resident"}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(args.cpu_tokens)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if code == B.DRK_BF16 else "f32", "data": "synthetic",
+            "config": {"workload": f"{wl.name}-shaped packed micro-batch", "T": T, "H": H, "V": V, "segments": S,
+                       "rollout_batch": f"{R} rollouts x {Tmax} turns", "mrs": args.mrs,
+                       "dW": args.dw_dtype, "dH": args.dh_dtype, "v_chunk": args.v_chunk or "default",
+                       "l2": "inputs exceed L2 (W alone is %.2f GB); no flush" % (V * H * 2 / 1e9),
+                       "parallelism": f"dp{world}: one micro-batch per rank, no collective on the loss path"},
+            "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s",
+                         "frac": achieved / peaks["tflops"], "traffic": None,
+                         "kernel": "umma_gemm_kernel (all four instantiations inside one drk_pg_loss_fwd_bwd call)",
+                         "flops_per_call": flops, "call_ms": fused_ms, "gemm_launches_per_call": n_gemm_launches,
+                         "peak_source": f"bf16_tflops_sustained of {peaks['source']}",
+                         "frac_of_burst": achieved / peaks["burst"], "frac_of_nominal_2250": achieved / 2250.0},
+            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": n_launch, "clocks": clocks,
+            "status_word": status, "counters": {"kept_tokens": counters[0], "masked_tokens": counters[1],
+                                                "kept_segments": counters[2], "vetoed_segments": counters[3]},
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

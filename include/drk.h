@@ -1,0 +1,169 @@
+/*
+ * drk — fused policy-gradient loss over the LM head for multi-turn RL
+ * (turn-level leave-one-out advantages + geometric mismatch rejection sampling).
+ *
+ * C ABI of libdrk.so.  Hand-written CUDA for sm_100a; one GPU per process.
+ *
+ * Conventions that hold for every entry point unless stated otherwise:
+ *   - "device" pointers are CUDA device pointers of the current device; "host"
+ *     pointers are ordinary host memory.  The caller owns every buffer, the
+ *     workspace included; the library allocates nothing and keeps no state
+ *     between calls apart from read-only per-process set-up (driver entry
+ *     points, kernel attributes).
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*, NULL =
+ *     the legacy default stream) and return without synchronising.  Scalar
+ *     results (loss, counters, status) stay in device memory.
+ *   - Return value: DRK_OK or a negative drk_status.  On a negative return
+ *     nothing was enqueued.  Conditions only the device can see set bits in the
+ *     device word `*status` (DRK_STATUS_*); no kernel traps or spins unbounded.
+ *   - All matrices are row-major and dense (leading dimension = row length).
+ *   - Row t of `hidden` predicts the token `ids[t]`; the caller has already
+ *     applied the next-token shift.
+ */
+#ifndef DRK_H_
+#define DRK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DRK_OK = 0,
+  DRK_ERR_INVALID_ARG = -1, /* null pointer, negative size, bad enum, misaligned pointer */
+  DRK_ERR_UNSUPPORTED = -2, /* shape outside what the kernels handle (see each call)     */
+  DRK_ERR_WORKSPACE = -3,   /* workspace_bytes smaller than drk_pg_workspace_bytes()     */
+  DRK_ERR_CUDA = -4,        /* a CUDA runtime or driver call failed                       */
+  DRK_ERR_ARCH = -5         /* current device is not compute capability 10.x             */
+} drk_status;
+
+typedef enum { DRK_F32 = 0, DRK_BF16 = 1 } drk_dtype;
+typedef enum { DRK_BASELINE_TRLOO = 0, DRK_BASELINE_GRPO = 1 } drk_baseline;
+typedef enum {
+  DRK_NORM_KEPT_TOKENS = 0,       /* scale = 1 / (loss-masked tokens of retained samples), >= 1 */
+  DRK_NORM_ALL_MASKED_TOKENS = 1, /* scale = 1 / (all loss-masked tokens inside segments), >= 1 */
+  DRK_NORM_EXPLICIT = 2           /* scale = explicit_scale                                      */
+} drk_norm;
+typedef enum {
+  DRK_ENGINE_AUTO = 0, /* bf16 inputs: tcgen05 tensor-core kernels; fp32 inputs: fp32 FFMA kernels */
+  DRK_ENGINE_SIMT = 1  /* force the FFMA kernels (exact fp32 products; slow; for cross-checks)     */
+} drk_engine;
+
+/* Bits of the device status word. */
+#define DRK_STATUS_BAD_ID 1u       /* some ids[t] outside [0,V): that row's target logit reads as 0 */
+#define DRK_STATUS_BAD_SEGMENTS 2u /* cu_seqlens not non-decreasing within [0,T]: segment skipped   */
+#define DRK_STATUS_NONFINITE 4u    /* a non-finite log-sum-exp was produced                         */
+#define DRK_STATUS_TIMEOUT 8u      /* a bounded on-chip wait expired; results are invalid           */
+
+/*
+ * Reward-to-go returns and turn-level advantages for a whole rollout batch
+ * (Sec. 4.2: Eq. 2 for the return, Eq. 5 for TRLOO, Eq. 3 for the GRPO mean
+ * baseline).
+ *
+ *   G[i,t]   = sum over valid t' >= t of gamma^(t'-t) * reward[i,t']
+ *   group    = rollouts j with prompt_of_rollout[j] == prompt_of_rollout[i] and valid[j,t]
+ *   TRLOO    : adv[i,t] = G[i,t] - mean_{j in group, j != i} G[j,t]   (0 when the group has one member)
+ *   GRPO     : adv[i,t] = G[i,t] - mean_{j in group} G[j,t]
+ *
+ * reward, valid, ret, adv, gsize are [R*Tmax] device arrays indexed i*Tmax+t;
+ * prompt_of_rollout is [R] device, non-decreasing (rollouts of a prompt are
+ * contiguous).  Invalid (i,t) get ret = adv = 0 and gsize = 0; valid ones get
+ * gsize = group size.  Arithmetic is fp64 inside, outputs are rounded to fp32.
+ * An all-equal group yields exactly 0.  R, Tmax >= 0 (0 enqueues nothing);
+ * Tmax <= 64, else DRK_ERR_UNSUPPORTED.  gamma must lie in [0,1].
+ */
+int drk_trloo_advantage(const float* reward, const uint8_t* valid,
+                        const int32_t* prompt_of_rollout, int32_t R, int32_t Tmax,
+                        float gamma, int32_t baseline, float* ret, float* adv,
+                        int32_t* gsize, void* stream);
+
+/* Parameters of the fused loss.  Fill with drk_pg_params_default() first. */
+typedef struct {
+  float mrs_lo;          /* Sec. 5.1: retain a sample iff mrs_lo <= w <= mrs_hi; default 0.999       */
+  float mrs_hi;          /* default 1.001; mrs_lo <= 0 drops the lower bound, +inf the upper one      */
+  float veto_ratio;      /* Sec. 5.1: reject if any token ratio < veto_ratio; default 1e-4; <=0 off   */
+  int32_t norm;          /* drk_norm; default DRK_NORM_KEPT_TOKENS                                   */
+  float explicit_scale;  /* used when norm == DRK_NORM_EXPLICIT                                      */
+  int32_t dw_dtype;      /* drk_dtype of dW; default DRK_F32                                         */
+  int32_t dh_dtype;      /* drk_dtype of dH; default DRK_F32                                         */
+  int32_t dw_accumulate; /* 0: dW = gradient; 1: dW += gradient (accumulation over micro-batches)    */
+  int32_t engine;        /* drk_engine; default DRK_ENGINE_AUTO                                      */
+  int32_t v_chunk;       /* vocabulary columns whose dLogits are held at once in the backward;
+                            0 = library default; rounded up to a multiple of 256                    */
+} drk_pg_params;
+
+void drk_pg_params_default(drk_pg_params* p); /* host pointer */
+
+/*
+ * Bytes of device workspace needed by drk_pg_logprob_fwd (which = 0) or
+ * drk_pg_loss_fwd_bwd (which = 1) for these sizes; p may be NULL for defaults
+ * (which = 0 ignores all of p but `engine`).  Returns 0 for invalid arguments.
+ * The workspace must be 256-byte aligned.
+ */
+size_t drk_pg_workspace_bytes(int64_t T, int32_t H, int32_t V, int32_t S, int32_t in_dtype,
+                              const drk_pg_params* p, int32_t which);
+
+/*
+ * Log-probability of the sampled token under the trainer's LM head, without
+ * materialising the logits: the quantity pi_train(a_t | s_t) of Sec. 5.1.
+ *
+ *   s[t,v]  = sum_h hidden[t,h] * W[v,h]
+ *   lse[t]  = log sum_v exp(s[t,v])         (running max / sum over vocabulary tiles)
+ *   logp[t] = s[t, ids[t]] - lse[t]
+ *
+ * hidden [T,H], W [V,H]: device, dtype in_dtype (both the same), 16-byte
+ * aligned; for DRK_BF16, H must be a multiple of 8.  ids [T] int32 device.
+ * logp, lse [T] float device.  status: device uint32, OR-ed into (the caller
+ * zeroes it).  engine: drk_engine.  T = 0 enqueues nothing.  T <= 2^24,
+ * 1 <= V <= 2^24, 1 <= H <= 65536.
+ */
+int drk_pg_logprob_fwd(const void* hidden, const void* W, int32_t in_dtype, const int32_t* ids,
+                       int64_t T, int32_t H, int32_t V, int32_t engine, float* logp, float* lse,
+                       void* workspace, size_t workspace_bytes, uint32_t* status, void* stream);
+
+/*
+ * Loss and gradients of one packed micro-batch: forward as above, geometric
+ * mismatch rejection sampling with token veto per training sample (Sec. 5.1),
+ * the REINFORCE surrogate with the caller's per-sample advantages (App. A,
+ * with TRLOO advantages per Sec. 4.2), and its gradient with the logits
+ * recomputed tile by tile.
+ *
+ *   segment g     = tokens [cu_seqlens[g], cu_seqlens[g+1]); its masked tokens M_g = {t: loss_mask[t] != 0}
+ *   delta_t       = logp[t] - rollout_logp[t]
+ *   seg_w[g]      = exp(mean_{t in M_g} delta_t)                  (1 if M_g is empty)
+ *   seg_keep[g]   = (ln lo <= mean delta <= ln hi) and (min_{M_g} delta_t >= ln veto) and M_g not empty
+ *   c_t           = seg_keep[g(t)] * mask_t * seg_adv[g(t)] * scale      (0 outside every segment)
+ *   loss          = - sum_t c_t * logp[t]
+ *   dL[t,v]       = c_t * (exp(s[t,v] - lse[t]) - [v == ids[t]])         (c_t is a constant)
+ *   dH[t,:]       = sum_v dL[t,v] * W[v,:]       dW[v,:] (+)= sum_t dL[t,v] * hidden[t,:]
+ *
+ * rollout_logp [T] float, loss_mask [T] uint8, cu_seqlens [S+1] int32
+ * (non-decreasing, within [0,T]), seg_adv [S] float: device.  Outputs, all
+ * device: loss [1] float; logp, lse [T]; seg_w [S] float; seg_keep [S] uint8;
+ * counters [4] int64 = {kept masked tokens, masked tokens in segments, kept
+ * segments, vetoed segments}; dH [T,H] of p->dh_dtype; dW [V,H] of
+ * p->dw_dtype.  dH and dW must be 16-byte aligned.  With bf16 inputs dL is
+ * rounded to bf16 before the two gradient contractions, which accumulate in
+ * fp32.  Rows with c_t = 0 get dH = 0 exactly.  S = 0 or T = 0: loss = 0,
+ * gradients 0 (dW untouched when accumulating).
+ */
+int drk_pg_loss_fwd_bwd(const void* hidden, const void* W, int32_t in_dtype, const int32_t* ids,
+                        const float* rollout_logp, const uint8_t* loss_mask,
+                        const int32_t* cu_seqlens, const float* seg_adv, int64_t T, int32_t H,
+                        int32_t V, int32_t S, const drk_pg_params* p, float* loss, float* logp,
+                        float* lse, float* seg_w, uint8_t* seg_keep, int64_t* counters, void* dH,
+                        void* dW, void* workspace, size_t workspace_bytes, uint32_t* status,
+                        void* stream);
+
+/* Number of kernels the last call on this host thread enqueued (0 after an error). */
+int drk_last_launch_count(void);
+
+const char* drk_status_string(int status);
+int drk_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DRK_H_ */

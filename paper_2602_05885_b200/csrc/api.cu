@@ -1,0 +1,258 @@
+// C-ABI entry points of libdrk.so: argument validation, workspace carving, dispatch.
+#include "common.cuh"
+#include <cmath>
+#include <limits>
+
+namespace drk {
+
+thread_local int g_launches = 0;
+
+namespace {
+
+constexpr int kDefaultVChunk = 8192;
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+int check_arch() {
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return DRK_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return DRK_ERR_CUDA;
+  return major == 10 ? DRK_OK : DRK_ERR_ARCH;
+}
+
+bool use_simt(int in_dtype, int engine) { return in_dtype == DRK_F32 || engine == DRK_ENGINE_SIMT; }
+
+bool sizes_ok(int64_t T, int H, int V, int in_dtype) {
+  if (T < 0 || T > (1 << 24) || H < 1 || H > 65536 || V < 1 || V > (1 << 24)) return false;
+  if (in_dtype != DRK_F32 && in_dtype != DRK_BF16) return false;
+  return true;
+}
+
+int round_vchunk(int v_chunk, int V) {
+  int vc = v_chunk > 0 ? v_chunk : kDefaultVChunk;
+  vc = (int)(ceil_div(vc, 256) * 256);
+  const int vmax = (int)(ceil_div(V, 256) * 256);
+  return vc < vmax ? vc : vmax;
+}
+
+// Carves 256-byte aligned pieces off the caller's workspace.
+struct Carver {
+  char* base;
+  size_t off = 0;
+  explicit Carver(void* b) : base(static_cast<char*>(b)) {}
+  void* take(size_t bytes) {
+    void* p = base ? base + off : nullptr;
+    off += align_up(bytes, 256);
+    return p;
+  }
+};
+
+struct FwdWs {
+  float* part;
+  float* tgt;
+  int nsplit;
+};
+FwdWs carve_fwd(Carver& c, int64_t T, int V, bool simt) {
+  FwdWs w;
+  w.nsplit = simt ? simt_nsplit(T, V) : umma_nsplit(T, V);
+  w.part = static_cast<float*>(c.take(sizeof(float) * 2 * (size_t)w.nsplit * (size_t)T));
+  w.tgt = static_cast<float*>(c.take(sizeof(float) * (size_t)T));
+  return w;
+}
+
+struct BwdWs {
+  float* coeff;
+  double* seg_stats;
+  void* dL;
+  float* dH_acc;
+  int vc;
+};
+BwdWs carve_bwd(Carver& c, int64_t T, int H, int V, int S, bool simt, const drk_pg_params& p) {
+  BwdWs w;
+  w.vc = round_vchunk(p.v_chunk, V);
+  w.coeff = static_cast<float*>(c.take(sizeof(float) * (size_t)T));
+  w.seg_stats = static_cast<double*>(c.take(sizeof(double) * 4 * (size_t)S));
+  w.dL = c.take((simt ? 4 : 2) * (size_t)T * (size_t)w.vc);
+  w.dH_acc = (p.dh_dtype == DRK_BF16) ? static_cast<float*>(c.take(sizeof(float) * (size_t)T * (size_t)H)) : nullptr;
+  return w;
+}
+
+bool params_ok(const drk_pg_params& p) {
+  if (p.norm < 0 || p.norm > 2) return false;
+  if (p.dw_dtype != DRK_F32 && p.dw_dtype != DRK_BF16) return false;
+  if (p.dh_dtype != DRK_F32 && p.dh_dtype != DRK_BF16) return false;
+  if (p.engine != DRK_ENGINE_AUTO && p.engine != DRK_ENGINE_SIMT) return false;
+  if (p.v_chunk < 0) return false;
+  if (std::isnan(p.mrs_lo) || std::isnan(p.mrs_hi) || std::isnan(p.veto_ratio)) return false;
+  if (p.norm == DRK_NORM_EXPLICIT && !std::isfinite(p.explicit_scale)) return false;
+  return true;
+}
+
+int run_fwd(const void* hidden, const void* W, int in_dtype, const int32_t* ids, int64_t T, int H, int V,
+            bool simt, const FwdWs& w, float* logp, float* lse, uint32_t* status, cudaStream_t st) {
+  if (simt) {
+    SimtFwdArgs a{hidden, W, in_dtype, ids, T, H, V, logp, lse, w.part, w.tgt, w.nsplit, status};
+    return launch_simt_fwd(a, st);
+  }
+  UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, w.part, w.tgt, w.nsplit, status};
+  return launch_umma_fwd(a, st);
+}
+
+}  // namespace
+}  // namespace drk
+
+using namespace drk;
+
+extern "C" {
+
+void drk_pg_params_default(drk_pg_params* p) {
+  if (!p) return;
+  p->mrs_lo = 0.999f;
+  p->mrs_hi = 1.001f;
+  p->veto_ratio = 1e-4f;
+  p->norm = DRK_NORM_KEPT_TOKENS;
+  p->explicit_scale = 1.0f;
+  p->dw_dtype = DRK_F32;
+  p->dh_dtype = DRK_F32;
+  p->dw_accumulate = 0;
+  p->engine = DRK_ENGINE_AUTO;
+  p->v_chunk = 0;
+}
+
+size_t drk_pg_workspace_bytes(int64_t T, int32_t H, int32_t V, int32_t S, int32_t in_dtype,
+                              const drk_pg_params* pp, int32_t which) {
+  drk_pg_params p;
+  if (pp) p = *pp; else drk_pg_params_default(&p);
+  if (!sizes_ok(T, H, V, in_dtype) || S < 0 || !params_ok(p) || (which != 0 && which != 1)) return 0;
+  const bool simt = use_simt(in_dtype, p.engine);
+  Carver c(nullptr);
+  carve_fwd(c, T, V, simt);
+  if (which == 1) carve_bwd(c, T, H, V, S, simt, p);
+  return c.off + 256;  // never 0 for valid arguments
+}
+
+int drk_trloo_advantage(const float* reward, const uint8_t* valid, const int32_t* prompt_of_rollout, int32_t R,
+                        int32_t Tmax, float gamma, int32_t baseline, float* ret, float* adv, int32_t* gsize,
+                        void* stream) {
+  g_launches = 0;
+  if (R < 0 || Tmax < 0) return DRK_ERR_INVALID_ARG;
+  if (baseline != DRK_BASELINE_TRLOO && baseline != DRK_BASELINE_GRPO) return DRK_ERR_INVALID_ARG;
+  if (!(gamma >= 0.f && gamma <= 1.f)) return DRK_ERR_INVALID_ARG;
+  if (Tmax > 64) return DRK_ERR_UNSUPPORTED;
+  if (R == 0 || Tmax == 0) return DRK_OK;
+  if (!reward || !valid || !prompt_of_rollout || !ret || !adv || !gsize) return DRK_ERR_INVALID_ARG;
+  int rc = check_arch();
+  if (rc != DRK_OK) return rc;
+  rc = launch_trloo(reward, valid, prompt_of_rollout, R, Tmax, gamma, baseline, ret, adv, gsize,
+                    static_cast<cudaStream_t>(stream));
+  if (rc != DRK_OK) g_launches = 0;
+  return rc;
+}
+
+int drk_pg_logprob_fwd(const void* hidden, const void* W, int32_t in_dtype, const int32_t* ids, int64_t T,
+                       int32_t H, int32_t V, int32_t engine, float* logp, float* lse, void* workspace,
+                       size_t workspace_bytes, uint32_t* status, void* stream) {
+  g_launches = 0;
+  if (!sizes_ok(T, H, V, in_dtype)) return DRK_ERR_INVALID_ARG;
+  if (engine != DRK_ENGINE_AUTO && engine != DRK_ENGINE_SIMT) return DRK_ERR_INVALID_ARG;
+  if (T == 0) return DRK_OK;
+  if (!hidden || !W || !ids || !logp || !lse || !workspace || !status) return DRK_ERR_INVALID_ARG;
+  if (!aligned(hidden, 16) || !aligned(W, 16) || !aligned(workspace, 256)) return DRK_ERR_INVALID_ARG;
+  const bool simt = use_simt(in_dtype, engine);
+  if (!simt && (H % 8) != 0) return DRK_ERR_UNSUPPORTED;
+  drk_pg_params p;
+  drk_pg_params_default(&p);
+  p.engine = engine;
+  if (workspace_bytes < drk_pg_workspace_bytes(T, H, V, 0, in_dtype, &p, 0)) return DRK_ERR_WORKSPACE;
+  int rc = check_arch();
+  if (rc != DRK_OK) return rc;
+  Carver c(workspace);
+  const FwdWs w = carve_fwd(c, T, V, simt);
+  rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, w, logp, lse, status, static_cast<cudaStream_t>(stream));
+  if (rc != DRK_OK) g_launches = 0;
+  return rc;
+}
+
+int drk_pg_loss_fwd_bwd(const void* hidden, const void* W, int32_t in_dtype, const int32_t* ids,
+                        const float* rollout_logp, const uint8_t* loss_mask, const int32_t* cu_seqlens,
+                        const float* seg_adv, int64_t T, int32_t H, int32_t V, int32_t S, const drk_pg_params* pp,
+                        float* loss, float* logp, float* lse, float* seg_w, uint8_t* seg_keep, int64_t* counters,
+                        void* dH, void* dW, void* workspace, size_t workspace_bytes, uint32_t* status,
+                        void* stream) {
+  g_launches = 0;
+  drk_pg_params p;
+  if (pp) p = *pp; else drk_pg_params_default(&p);
+  if (!sizes_ok(T, H, V, in_dtype) || S < 0 || S > (1 << 24) || !params_ok(p)) return DRK_ERR_INVALID_ARG;
+  if (!W || !dW || !loss || !counters || !workspace || !status) return DRK_ERR_INVALID_ARG;
+  if (T > 0 && (!hidden || !ids || !rollout_logp || !loss_mask || !logp || !lse || !dH)) return DRK_ERR_INVALID_ARG;
+  if (S > 0 && (!cu_seqlens || !seg_adv || !seg_w || !seg_keep)) return DRK_ERR_INVALID_ARG;
+  if (!aligned(hidden, 16) || !aligned(W, 16) || !aligned(dH, 16) || !aligned(dW, 16) || !aligned(workspace, 256) ||
+      !aligned(logp, 16) || !aligned(rollout_logp, 16) || !aligned(loss_mask, 4))
+    return DRK_ERR_INVALID_ARG;
+  const bool simt = use_simt(in_dtype, p.engine);
+  if (!simt && (H % 8) != 0) return DRK_ERR_UNSUPPORTED;
+  if (workspace_bytes < drk_pg_workspace_bytes(T, H, V, S, in_dtype, &p, 1)) return DRK_ERR_WORKSPACE;
+  int rc = check_arch();
+  if (rc != DRK_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  Carver c(workspace);
+  const FwdWs fw = carve_fwd(c, T, V, simt);
+  const BwdWs bw = carve_bwd(c, T, H, V, S, simt, p);
+
+  auto fail = [&](int code) { g_launches = 0; return code; };
+
+  if (T > 0) {
+    rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, fw, logp, lse, status, st);
+    if (rc != DRK_OK) return fail(rc);
+  }
+  MrsArgs m{};
+  m.logp = logp; m.rollout_logp = rollout_logp; m.loss_mask = loss_mask; m.cu = cu_seqlens; m.seg_adv = seg_adv;
+  m.T = T; m.S = S;
+  m.ln_lo = p.mrs_lo > 0.f ? std::log((double)p.mrs_lo) : -std::numeric_limits<double>::infinity();
+  m.ln_hi = std::isinf(p.mrs_hi) ? std::numeric_limits<double>::infinity() : std::log((double)p.mrs_hi);
+  m.ln_veto = p.veto_ratio > 0.f ? std::log((double)p.veto_ratio) : -std::numeric_limits<double>::infinity();
+  m.norm = p.norm; m.explicit_scale = p.explicit_scale;
+  m.seg_w = seg_w; m.seg_keep = seg_keep; m.loss = loss; m.counters = counters; m.coeff = bw.coeff;
+  m.seg_stats = bw.seg_stats; m.status = status;
+  rc = launch_mrs(m, st);
+  if (rc != DRK_OK) return fail(rc);
+
+  if (T == 0) {
+    // no tokens: gradients are zero
+    if (!p.dw_accumulate) {
+      const size_t esz = p.dw_dtype == DRK_BF16 ? 2 : 4;
+      if (cudaMemsetAsync(dW, 0, esz * (size_t)V * (size_t)H, st) != cudaSuccess) return fail(DRK_ERR_CUDA);
+    }
+    return DRK_OK;
+  }
+  if (simt) {
+    SimtBwdArgs b{hidden, W, in_dtype, ids, T, H, V, lse, bw.coeff, static_cast<float*>(bw.dL), bw.vc,
+                  dH, p.dh_dtype, bw.dH_acc, dW, p.dw_dtype, p.dw_accumulate};
+    rc = launch_simt_bwd(b, st);
+  } else {
+    UmmaBwdArgs b{hidden, W, ids, T, H, V, lse, bw.coeff, static_cast<__nv_bfloat16*>(bw.dL), bw.vc,
+                  dH, p.dh_dtype, bw.dH_acc, dW, p.dw_dtype, p.dw_accumulate, status};
+    rc = launch_umma_bwd(b, st);
+  }
+  if (rc != DRK_OK) return fail(rc);
+  return DRK_OK;
+}
+
+int drk_last_launch_count(void) { return g_launches; }
+
+const char* drk_status_string(int s) {
+  switch (s) {
+    case DRK_OK: return "ok";
+    case DRK_ERR_INVALID_ARG: return "invalid argument";
+    case DRK_ERR_UNSUPPORTED: return "unsupported shape";
+    case DRK_ERR_WORKSPACE: return "workspace too small";
+    case DRK_ERR_CUDA: return "CUDA call failed";
+    case DRK_ERR_ARCH: return "device is not sm_100";
+    default: return "unknown status";
+  }
+}
+
+int drk_version(void) { return 100; }
+
+}  // extern "C"

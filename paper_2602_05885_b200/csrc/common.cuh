@@ -1,0 +1,83 @@
+// Shared host/device helpers of the drk library (not part of the public ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "../../include/drk.h"
+
+namespace drk {
+
+// Per-thread count of kernels enqueued by the running entry point.
+extern thread_local int g_launches;
+
+#define DRK_CUDA_CHECK(expr)                      \
+  do {                                            \
+    cudaError_t e__ = (expr);                     \
+    if (e__ != cudaSuccess) return DRK_ERR_CUDA;  \
+  } while (0)
+
+// Call after every kernel launch: counts it and maps launch errors.
+#define DRK_LAUNCHED()                                  \
+  do {                                                  \
+    ++::drk::g_launches;                                \
+    if (cudaGetLastError() != cudaSuccess) return DRK_ERR_CUDA; \
+  } while (0)
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+template <typename T> __device__ __forceinline__ float to_f32(T x);
+template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// ---- internal launchers (each returns a drk_status) -------------------------------------------
+
+int launch_trloo(const float* reward, const uint8_t* valid, const int32_t* prompt, int R, int Tmax,
+                 float gamma, int baseline, float* ret, float* adv, int32_t* gsize, cudaStream_t st);
+
+// Per-segment statistics, rejection decision, coefficients and loss.
+struct MrsArgs {
+  const float* logp; const float* rollout_logp; const uint8_t* loss_mask; const int32_t* cu;
+  const float* seg_adv; int64_t T; int S;
+  double ln_lo, ln_hi, ln_veto; int norm; float explicit_scale;
+  float* seg_w; uint8_t* seg_keep; float* loss; int64_t* counters; float* coeff /*[T]*/;
+  double* seg_stats /*[S*4] workspace*/; uint32_t* status;
+};
+int launch_mrs(const MrsArgs& a, cudaStream_t st);
+
+// FFMA path.
+struct SimtFwdArgs {
+  const void* hidden; const void* W; int in_dtype; const int32_t* ids; int64_t T; int H; int V;
+  float* logp; float* lse; float* part /*[nsplit*T*2]*/; float* tgt /*[T]*/; int nsplit; uint32_t* status;
+};
+int simt_nsplit(int64_t T, int V);
+int launch_simt_fwd(const SimtFwdArgs& a, cudaStream_t st);
+int launch_lse_merge(const float* part, const float* tgt, const int32_t* ids, int64_t T, int V, int nsplit,
+                     float* logp, float* lse, uint32_t* status, cudaStream_t st);
+struct SimtBwdArgs {
+  const void* hidden; const void* W; int in_dtype; const int32_t* ids; int64_t T; int H; int V;
+  const float* lse; const float* coeff; float* dL /*[T*vc] fp32 workspace*/; int vc;
+  void* dH; int dh_dtype; float* dH_acc /*fp32 [T,H] or null when dH is fp32*/;
+  void* dW; int dw_dtype; int dw_accumulate;
+};
+int launch_simt_bwd(const SimtBwdArgs& a, cudaStream_t st);
+
+// tcgen05 path (bf16 inputs).
+struct UmmaFwdArgs {
+  const void* hidden; const void* W; const int32_t* ids; int64_t T; int H; int V;
+  float* logp; float* lse; float* part /*[nsplit*T*2]*/; float* tgt; int nsplit; uint32_t* status;
+};
+int umma_nsplit(int64_t T, int V);
+int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st);
+struct UmmaBwdArgs {
+  const void* hidden; const void* W; const int32_t* ids; int64_t T; int H; int V;
+  const float* lse; const float* coeff; __nv_bfloat16* dL /*[T*vc]*/; int vc;
+  void* dH; int dh_dtype; float* dH_acc; void* dW; int dw_dtype; int dw_accumulate; uint32_t* status;
+};
+int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st);
+
+// Small utility kernels.
+int launch_f32_to_bf16(const float* src, __nv_bfloat16* dst, size_t n, cudaStream_t st);
+
+}  // namespace drk

@@ -1,0 +1,569 @@
+// tcgen05 path of the fused LM-head loss (bf16 operands, fp32 accumulation in tensor memory).
+//
+// One persistent, warp-specialised GEMM kernel, instantiated for the four contractions of the path:
+//
+//   FWD : S = hidden W^T tile by tile; epilogue keeps a running (max, sum-exp) per row over the
+//         unit's vocabulary range and picks out the sampled token's logit.  Logits never leave
+//         the SM.
+//   DL  : the same tiles for one vocabulary chunk; epilogue stores
+//         dL = c_t (exp(s - lse_t) - onehot) as bf16 into the chunk buffer [T, vc].
+//   DW  : dW[chunk] (+)= dL^T hidden        (both operands have M/N contiguous: MN-major)
+//   DH  : dH (+)= dL W[chunk]               (A K-major, B MN-major)
+//
+// Tile 128 x 256 x 64, one CTA per SM, 192 threads:
+//   warp 0    : TMA producer (one lane): 128B-swizzled operand tiles into a 4-stage ring
+//   warp 1    : tensor-memory allocation; one lane issues tcgen05.mma (4 per stage, K = 16 each)
+//               into one of two 256-column fp32 accumulators and commits to mbarriers
+//   warps 2-5 : epilogue; warp w reads tensor-memory lanes 32*(w%4)..+31, one accumulator row per
+//               thread, 32 columns per tcgen05.ld, while the MMA warp fills the other accumulator
+// Every mbarrier wait is bounded; on expiry the block raises DRK_STATUS_TIMEOUT, drains its
+// in-flight copies and MMAs, frees tensor memory and returns.
+#include "common.cuh"
+#include "umma.cuh"
+#include <cuda.h>
+#include <math_constants.h>
+#include <mutex>
+
+namespace drk {
+
+namespace {
+
+constexpr int TM = 128, TN = 256, TK = 64, STAGES = 4;
+constexpr int A_BYTES = TM * TK * 2;  // 16 KiB
+constexpr int B_BYTES = TN * TK * 2;  // 32 KiB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int SUB_BYTES = 64 * TK * 2;  // one 64-wide MN-major box: 64 k-rows x 128 B
+constexpr int NUM_THREADS = 192;
+constexpr int NUM_BARS = 2 * STAGES + 5;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + NUM_BARS * 8 + 16;
+constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;  // 2 s: far above any legitimate wait
+constexpr uint64_t DRAIN_LIMIT_NS = 20000000ull;   // 20 ms per outstanding copy when giving up
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+enum Mode { FWD = 0, DL = 1, DW = 2, DH = 3 };
+
+struct UmmaParams {
+  int m_tiles, n_tiles, k_blocks, group_m, nj, tiles_per_unit, num_units;
+  int64_t rows;  // valid extent of the tile-row index (T, or the chunk's width for DW)
+  int cols;      // valid extent of the tile-column index (V, the chunk's width, or H)
+  int v0;        // first vocabulary column of the chunk (0 for FWD)
+  int64_t T;
+  const int32_t* ids;
+  const float* lse;
+  const float* coeff;
+  float* part;
+  float* tgt;
+  __nv_bfloat16* dL;
+  int vc;
+  void* C;
+  const void* C_in;
+  int64_t ldc;
+  int beta, out_bf16, in_bf16;
+  uint32_t* status;
+};
+
+struct Unit {
+  int m, j, n_begin, n_end;
+};
+
+__device__ __forceinline__ Unit decode_unit(const UmmaParams& p, int u) {
+  const int per_group = p.group_m * p.nj;
+  const int g = u / per_group;
+  const int rem = u - g * per_group;
+  const int gm = min(p.group_m, p.m_tiles - g * p.group_m);
+  Unit r;
+  r.j = rem / gm;
+  r.m = g * p.group_m + rem % gm;
+  r.n_begin = r.j * p.tiles_per_unit;
+  r.n_end = min(p.n_tiles, r.n_begin + p.tiles_per_unit);
+  return r;
+}
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Warp-collective bounded wait: all 32 lanes poll, and leave together.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort, int lane) {
+  uint64_t t0 = 0;
+  uint32_t polls = 0;
+#pragma unroll 1
+  for (;;) {
+    const bool done = ptx::mbar_try_wait(bar, parity);
+    if (__all_sync(0xffffffffu, done)) return true;
+    if ((++polls & 0x3ffu) == 0) {
+      if (t0 == 0) t0 = ptx::globaltimer_ns();
+      const bool give_up = (*abort != 0) || (ptx::globaltimer_ns() - t0 > WAIT_LIMIT_NS);
+      if (__any_sync(0xffffffffu, give_up)) {
+        if (lane == 0) *abort = 1;
+        return false;
+      }
+    }
+  }
+}
+
+// Store 32 consecutive fp32 results of one row, optionally added to what is there, as fp32 or bf16.
+__device__ __forceinline__ void store_row_chunk(const UmmaParams& p, int64_t row, int col, float (&x)[32]) {
+  const int64_t off = row * p.ldc + col;
+  const int nvalid = min(32, p.cols - col);
+  if (nvalid == 32) {
+    if (p.beta) {
+      if (p.in_bf16) {
+        const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.C_in) + off);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const uint4 w = src[q];
+          const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            x[q * 8 + e * 2 + 0] += __uint_as_float(ws[e] << 16);
+            x[q * 8 + e * 2 + 1] += __uint_as_float(ws[e] & 0xffff0000u);
+          }
+        }
+      } else {
+        const float4* src = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p.C_in) + off);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const float4 w = src[q];
+          x[q * 4 + 0] += w.x; x[q * 4 + 1] += w.y; x[q * 4 + 2] += w.z; x[q * 4 + 3] += w.w;
+        }
+      }
+    }
+    if (p.out_bf16) {
+      uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.C) + off);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        dst[q] = make_uint4(pack_bf16(x[q * 8 + 0], x[q * 8 + 1]), pack_bf16(x[q * 8 + 2], x[q * 8 + 3]),
+                            pack_bf16(x[q * 8 + 4], x[q * 8 + 5]), pack_bf16(x[q * 8 + 6], x[q * 8 + 7]));
+    } else {
+      float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.C) + off);
+#pragma unroll
+      for (int q = 0; q < 8; ++q) dst[q] = make_float4(x[q * 4 + 0], x[q * 4 + 1], x[q * 4 + 2], x[q * 4 + 3]);
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      if (j < nvalid) {
+        float v = x[j];
+        if (p.beta)
+          v += p.in_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.C_in)[off + j])
+                         : reinterpret_cast<const float*>(p.C_in)[off + j];
+        if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.C)[off + j] = __float2bfloat16(v);
+        else reinterpret_cast<float*>(p.C)[off + j] = v;
+      }
+    }
+  }
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                 const UmmaParams p) {
+  constexpr bool A_MN = (MODE == DW);
+  constexpr bool B_MN = (MODE == DW || MODE == DH);
+  constexpr uint32_t IDESC = ptx::make_idesc_bf16(TM, TN, A_MN ? 1 : 0, B_MN ? 1 : 0);
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = ptx::smem_u32(smem_raw);
+  const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
+  uint8_t* smem = smem_raw + pad;
+  const uint32_t smem_base = raw_addr + pad;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+  const uint32_t done_bar = bar_base + 8u * (2 * STAGES + 4);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NUM_BARS);
+  volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(full_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(tfull_bar(a), 1);
+      ptx::mbar_init(tempty_bar(a), 4);
+    }
+    ptx::mbar_init(done_bar, 1);
+    *abort = 0;
+    ptx::fence_barrier_init();
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(ptx::smem_u32(tmem_slot), 512);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      ptx::prefetch_tensormap(&tmA);
+      ptx::prefetch_tensormap(&tmB);
+      uint32_t it = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < p.num_units && ok; u += gridDim.x) {
+        const Unit un = decode_unit(p, u);
+        for (int n = un.n_begin; n < un.n_end && ok; ++n) {
+          for (int kb = 0; kb < p.k_blocks; ++kb) {
+            const int s = it % STAGES;
+            const uint32_t ph = (it / STAGES) & 1u;
+            if (!ptx::mbar_wait(empty_bar(s), ph ^ 1u, abort, WAIT_LIMIT_NS)) { ok = false; break; }
+            ptx::mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES);
+            const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
+            if constexpr (MODE == FWD || MODE == DL) {
+              ptx::tma_load_2d(sa, &tmA, full_bar(s), kb * TK, un.m * TM);
+              ptx::tma_load_2d(sb, &tmB, full_bar(s), kb * TK, p.v0 + n * TN);
+            } else if constexpr (MODE == DW) {
+#pragma unroll
+              for (int j = 0; j < TM / 64; ++j)
+                ptx::tma_load_2d(sa + j * SUB_BYTES, &tmA, full_bar(s), un.m * TM + 64 * j, kb * TK);
+#pragma unroll
+              for (int j = 0; j < TN / 64; ++j)
+                ptx::tma_load_2d(sb + j * SUB_BYTES, &tmB, full_bar(s), n * TN + 64 * j, kb * TK);
+            } else {  // DH
+              ptx::tma_load_2d(sa, &tmA, full_bar(s), kb * TK, un.m * TM);
+#pragma unroll
+              for (int j = 0; j < TN / 64; ++j)
+                ptx::tma_load_2d(sb + j * SUB_BYTES, &tmB, full_bar(s), n * TN + 64 * j, p.v0 + kb * TK);
+            }
+            ++it;
+          }
+        }
+      }
+      if (!ok) {
+        // wait (bounded) for the copies still in flight before the block leaves
+        const uint32_t first = it > STAGES ? it - STAGES : 0;
+        for (uint32_t j = first; j < it; ++j)
+          ptx::mbar_wait(full_bar(j % STAGES), (j / STAGES) & 1u, nullptr, DRAIN_LIMIT_NS);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t it = 0, tc = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < p.num_units && ok; u += gridDim.x) {
+        const Unit un = decode_unit(p, u);
+        for (int n = un.n_begin; n < un.n_end && ok; ++n) {
+          const int acc = tc & 1;
+          const uint32_t aph = (tc >> 1) & 1u;
+          if (!ptx::mbar_wait(tempty_bar(acc), aph ^ 1u, abort, WAIT_LIMIT_NS)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t d_tmem = tmem_base + acc * TN;
+          for (int kb = 0; kb < p.k_blocks; ++kb) {
+            const int s = it % STAGES;
+            const uint32_t ph = (it / STAGES) & 1u;
+            if (!ptx::mbar_wait(full_bar(s), ph, abort, WAIT_LIMIT_NS)) { ok = false; break; }
+            ptx::tc_fence_after();
+            const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
+#pragma unroll
+            for (int k = 0; k < TK / 16; ++k) {
+              // K-major: 16 elements = 32 B further along the swizzled 128 B row.
+              // MN-major: 16 k-rows of 128 B = two 8-row swizzle atoms further.
+              const uint64_t da = A_MN ? ptx::make_smem_desc(sa + k * 2048, SUB_BYTES, 1024)
+                                       : ptx::make_smem_desc(sa + k * 32, 16, 1024);
+              const uint64_t db = B_MN ? ptx::make_smem_desc(sb + k * 2048, SUB_BYTES, 1024)
+                                       : ptx::make_smem_desc(sb + k * 32, 16, 1024);
+              ptx::mma_bf16_ss(d_tmem, da, db, IDESC, (kb | k) != 0 ? 1u : 0u);
+            }
+            ptx::mma_commit(empty_bar(s));  // frees the stage once these MMAs have read it
+            ++it;
+          }
+          if (!ok) break;
+          ptx::mma_commit(tfull_bar(acc));  // accumulator complete
+          ++tc;
+        }
+      }
+      if (!ok) {
+        ptx::mma_commit(done_bar);
+        ptx::mbar_wait(done_bar, 0, nullptr, DRAIN_LIMIT_NS);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int q = warp & 3;  // tensor-memory lane quarter this warp may read
+    uint32_t tc = 0;
+    bool ok = true;
+    for (int u = blockIdx.x; u < p.num_units && ok; u += gridDim.x) {
+      const Unit un = decode_unit(p, u);
+      const int64_t row = (int64_t)un.m * TM + q * 32 + lane;
+      const bool row_ok = row < p.rows;
+      // per-unit state
+      float run_m = -CUDART_INF_F, run_l = 0.f;  // FWD: log2-domain running max, sum
+      int id = -1;
+      float c_t = 0.f, z2 = 0.f;
+      if constexpr (MODE == FWD || MODE == DL) {
+        if (row_ok) id = p.ids[row];
+      }
+      if constexpr (MODE == DL) {
+        if (row_ok) { c_t = p.coeff[row]; z2 = p.lse[row] * kLog2e; }
+      }
+      for (int n = un.n_begin; n < un.n_end; ++n) {
+        const int acc = tc & 1;
+        const uint32_t aph = (tc >> 1) & 1u;
+        if (!mbar_wait_warp(tfull_bar(acc), aph, abort, lane)) { ok = false; break; }
+        ptx::tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * TN;
+#pragma unroll 1
+        for (int c = 0; c < TN / 32; ++c) {
+          uint32_t raw[32];
+          __syncwarp();
+          ptx::tmem_ld_32x32(taddr + c * 32, raw);
+          ptx::tmem_ld_wait();
+          float x[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(raw[j]);
+          const int col = n * TN + c * 32;  // column index within [0, cols)
+          if constexpr (MODE == FWD) {
+            if (col + 32 > p.cols) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (col + j >= p.cols) x[j] = -CUDART_INF_F;
+            }
+            if ((uint32_t)(id - col) < 32u) {
+              const int w = id - col;
+              float tg = 0.f;
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (j == w) tg = x[j];
+              p.tgt[row] = tg;
+            }
+            float cm = x[0];
+#pragma unroll
+            for (int j = 1; j < 32; ++j) cm = fmaxf(cm, x[j]);
+            const float m_new = fmaxf(run_m, cm * kLog2e);
+            if (m_new > -CUDART_INF_F) {
+              float s = 0.f;
+#pragma unroll
+              for (int j = 0; j < 32; ++j) s += ex2(fmaf(x[j], kLog2e, -m_new));
+              run_l = run_l * ex2(run_m - m_new) + s;
+              run_m = m_new;
+            }
+          } else if constexpr (MODE == DL) {
+            if (row_ok && col < p.cols) {
+              const int gcol = p.v0 + col;
+              if (c_t != 0.f) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                  const float pr = ex2(fmaf(x[j], kLog2e, -z2));
+                  x[j] = c_t * (pr - ((gcol + j == id) ? 1.f : 0.f));
+                }
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) x[j] = 0.f;
+              }
+              __nv_bfloat16* dst = p.dL + row * p.vc + col;
+              if (col + 32 <= p.cols) {
+                uint4* d4 = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+                for (int qd = 0; qd < 4; ++qd)
+                  d4[qd] = make_uint4(pack_bf16(x[qd * 8 + 0], x[qd * 8 + 1]), pack_bf16(x[qd * 8 + 2], x[qd * 8 + 3]),
+                                      pack_bf16(x[qd * 8 + 4], x[qd * 8 + 5]), pack_bf16(x[qd * 8 + 6], x[qd * 8 + 7]));
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                  if (col + j < p.cols) dst[j] = __float2bfloat16(x[j]);
+              }
+            }
+          } else {  // DW, DH
+            if (row_ok && col < p.cols) store_row_chunk(p, row, col, x);
+          }
+        }
+        // this warp has drained its quarter of the accumulator
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+        ++tc;
+      }
+      if (!ok) break;
+      if constexpr (MODE == FWD) {
+        if (row_ok) {
+          float* dst = p.part + ((int64_t)un.j * p.T + row) * 2;
+          dst[0] = run_m * kLn2;  // natural-log units, as the merge kernel expects
+          dst[1] = run_l;
+        }
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort) atomicOr(p.status, DRK_STATUS_TIMEOUT);
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  });
+  return fn;
+}
+
+// Row-major bf16 matrix [outer, inner] with row pitch `pitch_elems`; box = box_inner x box_outer,
+// 128-byte swizzle, zero fill outside the extents.
+bool make_map(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, uint64_t pitch_elems,
+              uint32_t box_inner, uint32_t box_outer) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {pitch_elems * 2};
+  cuuint32_t box[2] = {box_inner, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+  return n;
+}
+
+template <int MODE>
+int launch_mode(const CUtensorMap& a, const CUtensorMap& b, UmmaParams p, cudaStream_t st) {
+  p.num_units = p.m_tiles * p.nj;
+  if (p.num_units <= 0) return DRK_OK;
+  DRK_CUDA_CHECK(cudaFuncSetAttribute(umma_gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+  const int grid = p.num_units < sm_count() ? p.num_units : sm_count();
+  umma_gemm_kernel<MODE><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(a, b, p);
+  DRK_LAUNCHED();
+  return DRK_OK;
+}
+
+}  // namespace
+
+int umma_nsplit(int64_t T, int V) {
+  const int64_t m_tiles = ceil_div(T, TM);
+  const int n_tiles = (int)ceil_div(V, TN);
+  if (m_tiles <= 0) return 1;
+  const int sms = 148;
+  int best = 1;
+  double best_eff = -1.0;
+  for (int ns = 1; ns <= 32 && ns <= n_tiles; ++ns) {
+    const int per = (int)ceil_div(n_tiles, ns);
+    const int ns_eff = (int)ceil_div(n_tiles, per);
+    if (ns_eff != ns) continue;
+    if (per < 4 && ns > 1) continue;
+    const int64_t units = m_tiles * ns;
+    const int64_t waves = ceil_div(units, sms);
+    // time ~ waves * per tiles; work = m_tiles * n_tiles tiles
+    const double eff = (double)(m_tiles * (int64_t)n_tiles) / ((double)waves * per * sms);
+    if (eff > best_eff + 0.005) { best_eff = eff; best = ns; }
+  }
+  return best;
+}
+
+int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st) {
+  CUtensorMap mh, mw;
+  if (!make_map(&mh, a.hidden, a.H, a.T, a.H, TK, TM)) return DRK_ERR_CUDA;
+  if (!make_map(&mw, a.W, a.H, a.V, a.H, TK, TN)) return DRK_ERR_CUDA;
+  UmmaParams p{};
+  p.m_tiles = (int)ceil_div(a.T, TM);
+  p.n_tiles = (int)ceil_div(a.V, TN);
+  p.k_blocks = (int)ceil_div(a.H, TK);
+  p.nj = a.nsplit;
+  p.tiles_per_unit = (int)ceil_div(p.n_tiles, a.nsplit);
+  p.group_m = 148 / a.nsplit > 0 ? 148 / a.nsplit : 1;
+  p.rows = a.T; p.cols = a.V; p.v0 = 0; p.T = a.T;
+  p.ids = a.ids; p.part = a.part; p.tgt = a.tgt; p.status = a.status;
+  int rc = launch_mode<FWD>(mh, mw, p, st);
+  if (rc != DRK_OK) return rc;
+  return launch_lse_merge(a.part, a.tgt, a.ids, a.T, a.V, a.nsplit, a.logp, a.lse, a.status, st);
+}
+
+int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {
+  CUtensorMap mh_k, mw_k, mh_mn, mw_mn;
+  if (!make_map(&mh_k, a.hidden, a.H, a.T, a.H, TK, TM)) return DRK_ERR_CUDA;
+  if (!make_map(&mw_k, a.W, a.H, a.V, a.H, TK, TN)) return DRK_ERR_CUDA;
+  if (!make_map(&mh_mn, a.hidden, a.H, a.T, a.H, 64, TK)) return DRK_ERR_CUDA;
+  if (!make_map(&mw_mn, a.W, a.H, a.V, a.H, 64, TK)) return DRK_ERR_CUDA;
+  float* dh_acc = (a.dh_dtype == DRK_F32) ? (float*)a.dH : a.dH_acc;
+  const int n_chunks = (int)ceil_div(a.V, a.vc);
+  int chunk = 0;
+  for (int v0 = 0; v0 < a.V; v0 += a.vc, ++chunk) {
+    const int vc_this = a.V - v0 < a.vc ? a.V - v0 : a.vc;
+    CUtensorMap mdl_k, mdl_mn;
+    if (!make_map(&mdl_k, a.dL, vc_this, a.T, a.vc, TK, TM)) return DRK_ERR_CUDA;
+    if (!make_map(&mdl_mn, a.dL, vc_this, a.T, a.vc, 64, TK)) return DRK_ERR_CUDA;
+    {  // dL chunk = c (softmax - onehot), recomputed from hidden W^T
+      UmmaParams p{};
+      p.m_tiles = (int)ceil_div(a.T, TM);
+      p.n_tiles = (int)ceil_div(vc_this, TN);
+      p.k_blocks = (int)ceil_div(a.H, TK);
+      p.nj = p.n_tiles; p.tiles_per_unit = 1; p.group_m = 16;
+      p.rows = a.T; p.cols = vc_this; p.v0 = v0; p.T = a.T;
+      p.ids = a.ids; p.lse = a.lse; p.coeff = a.coeff; p.dL = a.dL; p.vc = a.vc; p.status = a.status;
+      int rc = launch_mode<DL>(mh_k, mw_k, p, st);
+      if (rc != DRK_OK) return rc;
+    }
+    {  // dW[v0 : v0 + vc_this, :] (+)= dL^T hidden
+      UmmaParams p{};
+      p.m_tiles = (int)ceil_div(vc_this, TM);
+      p.n_tiles = (int)ceil_div(a.H, TN);
+      p.k_blocks = (int)ceil_div(a.T, TK);
+      p.nj = p.n_tiles; p.tiles_per_unit = 1; p.group_m = 16;
+      p.rows = vc_this; p.cols = a.H; p.v0 = v0; p.T = a.T;
+      const size_t esz = a.dw_dtype == DRK_BF16 ? 2 : 4;
+      p.C = (char*)a.dW + (size_t)v0 * a.H * esz; p.C_in = p.C; p.ldc = a.H;
+      p.beta = a.dw_accumulate; p.out_bf16 = a.dw_dtype == DRK_BF16; p.in_bf16 = p.out_bf16;
+      p.status = a.status;
+      int rc = launch_mode<DW>(mdl_mn, mh_mn, p, st);
+      if (rc != DRK_OK) return rc;
+    }
+    {  // dH (+)= dL W[v0 : v0 + vc_this, :]
+      UmmaParams p{};
+      p.m_tiles = (int)ceil_div(a.T, TM);
+      p.n_tiles = (int)ceil_div(a.H, TN);
+      p.k_blocks = (int)ceil_div(vc_this, TK);
+      p.nj = p.n_tiles; p.tiles_per_unit = 1; p.group_m = 8;
+      p.rows = a.T; p.cols = a.H; p.v0 = v0; p.T = a.T;
+      const bool last = (chunk == n_chunks - 1);
+      p.C_in = dh_acc; p.in_bf16 = 0; p.ldc = a.H; p.beta = chunk > 0;
+      if (last && a.dh_dtype == DRK_BF16) { p.C = a.dH; p.out_bf16 = 1; }
+      else { p.C = dh_acc; p.out_bf16 = 0; }
+      p.status = a.status;
+      int rc = launch_mode<DH>(mdl_k, mw_mn, p, st);
+      if (rc != DRK_OK) return rc;
+    }
+  }
+  return DRK_OK;
+}
+
+}  // namespace drk

@@ -63,8 +63,8 @@ def rollout_batch(P: int, K: int, Tmax: int, len_lo: int, len_hi: int, seed: int
     ragged=False: every rollout is valid at every turn.
     ragged=True : rollout i ends after turn tau_i ~ U{1..Tmax}; in addition the
     first prompt keeps a single rollout alive at the last turn (a group of
-    one), the second prompt's rewards are all equal, and the third prompt's
-    rewards are all zero (where those prompts exist).
+    one), the second prompt's rollouts all run to the end with equal rewards,
+    and the third prompt's rewards are all zero (where those prompts exist).
     ctx_frac: fraction of each training sample that is unmasked context
     (prompt / feedback tokens) packed in front of the response.
     """
@@ -79,7 +79,8 @@ def rollout_batch(P: int, K: int, Tmax: int, len_lo: int, len_hi: int, seed: int
         # a group of size one at the last turn of prompt 0
         valid[0:K, Tmax - 1] = 0
         valid[0, :] = 1
-        if P > 1:   # all-equal, non-zero rewards
+        if P > 1:   # all-equal, non-zero rewards on rollouts that all run to the last turn
+            valid[K:2 * K, :] = 1
             reward[K:2 * K, :] = 1.25
         if P > 2:   # all-zero rewards
             reward[2 * K:3 * K, :] = 0.0

@@ -1,0 +1,212 @@
+"""Shared test machinery: builds seeded cases, runs the oracle on them, compares device results.
+
+The oracle side and the device side meet only here: both receive the same input arrays, and
+expected values always come from `oracle/`.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+from typing import Dict, Optional
+
+import numpy as np
+import torch
+
+from oracle import drk_oracle as O
+from paper_2602_05885_b200 import synth
+
+# Tolerances (per-token log-prob, loss, gradients, advantages) as stated for the method's target.
+TOL_LOGP_BF16 = 2e-3
+TOL_LOGP_F32 = 1e-4
+TOL_LOSS_REL = 1e-3
+TOL_GRAD_FRO = 1e-2
+TOL_ADV_REL = 1e-6
+
+
+def f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().cpu().to(torch.float64).numpy()
+
+
+@dataclass
+class Case:
+    name: str
+    dtype: torch.dtype
+    hidden: torch.Tensor          # [T,H] cpu, dtype
+    W: torch.Tensor               # [V,H] cpu, dtype
+    ids: torch.Tensor             # [T] int32
+    rollout_logp: torch.Tensor    # [T] float32
+    loss_mask: torch.Tensor       # [T] uint8
+    cu: torch.Tensor              # [S+1] int32
+    seg_rollout: torch.Tensor
+    seg_turn: torch.Tensor
+    rb: Optional[synth.RolloutBatch]
+    seg_adv: torch.Tensor         # [S] float32 (from the oracle's TRLOO unless given)
+    # oracle intermediates, computed once
+    s: np.ndarray = field(repr=False, default=None)
+    logp: np.ndarray = field(repr=False, default=None)
+    lse: np.ndarray = field(repr=False, default=None)
+
+    @property
+    def T(self):
+        return self.hidden.shape[0]
+
+    @property
+    def H(self):
+        return self.hidden.shape[1]
+
+    @property
+    def V(self):
+        return self.W.shape[0]
+
+    @property
+    def S(self):
+        return self.cu.shape[0] - 1
+
+
+def sample_ids_from_policy(s: np.ndarray, u: np.ndarray) -> np.ndarray:
+    """Inverse-CDF sampling of one token per row from softmax(s) with the given uniforms."""
+    lse = O.logsumexp_rows(s)
+    ids = np.empty(s.shape[0], dtype=np.int64)
+    for t in range(s.shape[0]):
+        cdf = np.cumsum(np.exp(s[t] - lse[t]))
+        ids[t] = min(int(np.searchsorted(cdf, u[t] * cdf[-1], side="right")), s.shape[1] - 1)
+    return ids
+
+
+def oracle_advantages(rb: synth.RolloutBatch, gamma: float = 1.0):
+    G = O.returns(rb.reward.numpy(), rb.valid.numpy(), gamma)
+    A, N = O.trloo_advantage(G, rb.valid.numpy(), rb.prompt_of_rollout.numpy())
+    return G, A, N
+
+
+def build_case(name: str, *, H: int, V: int, dtype: torch.dtype, P: int, K: int, Tmax: int,
+               len_lo: int, len_hi: int, capacity: int, seed: int, sigma: float = 0.05,
+               ragged: bool = False, ctx_frac: float = 0.0, outlier_frac: float = 0.0,
+               lead_pad: int = 0, microbatch: int = 0, uniform_ids: bool = False) -> Case:
+    rb = synth.rollout_batch(P, K, Tmax, len_lo, len_hi, seed, ragged=ragged, ctx_frac=ctx_frac)
+    plans = synth.pack_first_fit(rb, capacity - lead_pad)
+    plan = plans[microbatch]
+    plan.T = capacity
+    cu, mask, seg_rollout, seg_turn = synth.plan_tensors(plan, lead_pad=lead_pad)
+    T = capacity
+    hidden, W, _ = synth.dense_operands(T, H, V, dtype, seed + 1, "cpu")
+    S = cu.shape[0] - 1
+    outl = synth.pick_outlier_segments(S, 0.1, seed + 3) if outlier_frac > 0 else None
+    u, noise = synth.token_draws(T, seed + 2, "cpu", sigma=sigma, outlier_frac=outlier_frac,
+                                 outlier_segments=outl, cu_seqlens=cu)
+    s = O.logits(f64(hidden), f64(W))
+    if uniform_ids:
+        ids = synth.uniform_ids(T, V, seed + 4).numpy().astype(np.int64)
+    else:
+        ids = sample_ids_from_policy(s, u.numpy())
+    logp, lse = O.token_logprob(s, ids)
+    rollout_logp = torch.from_numpy((logp + noise.numpy().astype(np.float64)).astype(np.float32))
+    _, A, _ = oracle_advantages(rb)
+    seg_adv = torch.from_numpy(A[seg_rollout.numpy(), seg_turn.numpy()].astype(np.float32))
+    return Case(name, dtype, hidden, W, torch.from_numpy(ids.astype(np.int32)), rollout_logp, mask, cu,
+                seg_rollout, seg_turn, rb, seg_adv, s=s, logp=logp, lse=lse)
+
+
+def build_plain_case(name: str, *, T: int, H: int, V: int, dtype: torch.dtype, S: int, seed: int,
+                     sigma: float = 0.05, mask_frac: float = 0.0) -> Case:
+    """A case without rollout structure: S equal segments over all T tokens, advantages ~ N(0,1)."""
+    hidden, W, _ = synth.dense_operands(T, H, V, dtype, seed + 1, "cpu")
+    g = torch.Generator().manual_seed(seed)
+    S = min(S, T) if T > 0 else S
+    bounds = torch.linspace(0, T, S + 1).round().to(torch.int32)
+    mask = (torch.rand(T, generator=g) >= mask_frac).to(torch.uint8)
+    u, noise = synth.token_draws(T, seed + 2, "cpu", sigma=sigma)
+    s = O.logits(f64(hidden), f64(W))
+    ids = sample_ids_from_policy(s, u.numpy()) if T > 0 else np.zeros(0, dtype=np.int64)
+    logp, lse = O.token_logprob(s, ids) if T > 0 else (np.zeros(0), np.zeros(0))
+    rollout_logp = torch.from_numpy((logp + noise.numpy().astype(np.float64)).astype(np.float32))
+    seg_adv = torch.randn(S, generator=g).float()
+    z = torch.zeros(S, dtype=torch.int64)
+    return Case(name, dtype, hidden, W, torch.from_numpy(ids.astype(np.int32)), rollout_logp, mask, bounds,
+                z, z, None, seg_adv, s=s, logp=logp, lse=lse)
+
+
+# ---------------------------------------------------------------------------
+# Oracle evaluation of a case under given MRS parameters
+# ---------------------------------------------------------------------------
+
+def wide_band(case: Case):
+    """(lo, hi) = exp(-+q) with q the oracle's median |mean delta|: about half the samples pass."""
+    m = O.mrs(case.logp, f64(case.rollout_logp), case.loss_mask.numpy(), case.cu.numpy(), lo=0.0, hi=math.inf)
+    nz = m.n_masked > 0
+    q = float(np.median(np.abs(m.mean_delta[nz]))) if nz.any() else 1e-3
+    return float(np.float32(math.exp(-q))), float(np.float32(math.exp(q)))
+
+
+def oracle_eval(case: Case, lo: float, hi: float, veto: float, norm: int = 0, explicit_scale: float = 1.0,
+                keep_override=None, seg_adv=None, want_grads: bool = True) -> Dict:
+    """lo, hi, veto must already be float32-representable (the C ABI takes floats)."""
+    m = O.mrs(case.logp, f64(case.rollout_logp), case.loss_mask.numpy(), case.cu.numpy(), lo, hi, veto)
+    keep = m.keep if keep_override is None else np.asarray(keep_override).astype(bool)
+    adv = f64(case.seg_adv) if seg_adv is None else np.asarray(seg_adv, dtype=np.float64)
+    lr = O.coeff_and_loss(case.logp, keep, case.loss_mask.numpy(), case.cu.numpy(), adv, norm, explicit_scale)
+    out = dict(mrs=m, keep=keep, coeff=lr.coeff, loss=lr.loss, kept_tokens=lr.kept_tokens,
+               masked_tokens=lr.masked_tokens, kept_segs=lr.kept_segs, vetoed_segs=int(m.vetoed.sum()))
+    if want_grads:
+        dH, dW = O.gradients(f64(case.hidden), f64(case.W), case.s, case.lse, case.ids.numpy(), lr.coeff)
+        out["dH"], out["dW"] = dH, dW
+    return out
+
+
+def ambiguous_segments(m: O.MrsResult, lo: float, hi: float, veto: float, tol_mean: float, tol_tok: float):
+    """Segments whose decision lies within rounding distance of a threshold: either answer is right."""
+    ln_lo = math.log(lo) if lo > 0 else -math.inf
+    ln_hi = math.log(hi) if math.isfinite(hi) else math.inf
+    ln_veto = math.log(veto) if veto > 0 else -math.inf
+    amb = (np.abs(m.mean_delta - ln_lo) < tol_mean) | (np.abs(m.mean_delta - ln_hi) < tol_mean) | \
+          (np.abs(m.min_delta - ln_veto) < tol_tok)
+    return amb & (m.n_masked > 0)
+
+
+def rel_fro(a: np.ndarray, b: np.ndarray) -> float:
+    nb = float(np.linalg.norm(b))
+    if nb == 0.0:
+        return 0.0 if float(np.abs(a).max(initial=0.0)) == 0.0 else math.inf
+    return float(np.linalg.norm(a - b)) / nb
+
+
+def check_against_oracle(case: Case, dev: Dict, lo: float, hi: float, veto: float, norm: int = 0,
+                         explicit_scale: float = 1.0, seg_adv=None, dW_before: Optional[np.ndarray] = None):
+    """dev: dict of CPU tensors from the device path (logp, lse, seg_w, seg_keep, loss, counters, dH, dW)."""
+    tol_logp = TOL_LOGP_F32 if case.dtype == torch.float32 else TOL_LOGP_BF16
+    T, S = case.T, case.S
+    if T > 0:
+        err = np.abs(f64(dev["logp"]) - case.logp).max()
+        assert err <= tol_logp, f"logp max err {err}"
+        err = np.abs(f64(dev["lse"]) - case.lse).max()
+        assert err <= tol_logp, f"lse max err {err}"
+    first = oracle_eval(case, lo, hi, veto, norm, explicit_scale, seg_adv=seg_adv, want_grads=False)
+    m = first["mrs"]
+    keep_dev = dev["seg_keep"].numpy().astype(bool)
+    amb = ambiguous_segments(m, lo, hi, veto, tol_mean=tol_logp, tol_tok=tol_logp)
+    mismatch = (keep_dev != m.keep) & ~amb
+    assert not mismatch.any(), f"keep differs on unambiguous segments {np.nonzero(mismatch)[0]}"
+    ref = oracle_eval(case, lo, hi, veto, norm, explicit_scale, keep_override=keep_dev, seg_adv=seg_adv)
+    if S > 0:
+        nz = m.n_masked > 0
+        werr = np.abs(f64(dev["seg_w"]) - m.w)[nz] / m.w[nz]
+        assert werr.max(initial=0.0) <= 2 * tol_logp, f"seg_w rel err {werr.max()}"
+        assert (f64(dev["seg_w"])[~nz] == 1.0).all()
+    counters = dev["counters"].numpy()
+    assert counters[0] == ref["kept_tokens"] and counters[1] == ref["masked_tokens"]
+    assert counters[2] == ref["kept_segs"]
+    if not amb.any():
+        assert counters[3] == ref["vetoed_segs"]
+    # loss: relative to max(|loss|, 1e-3 * sum |c_t logp_t|) since advantages cancel inside groups
+    denom = max(abs(ref["loss"]), 1e-3 * float(np.sum(np.abs(ref["coeff"] * case.logp))), 1e-30)
+    lerr = abs(float(dev["loss"]) - ref["loss"]) / denom
+    assert lerr <= TOL_LOSS_REL or abs(float(dev["loss"]) - ref["loss"]) < 1e-7, f"loss rel err {lerr}"
+    dH = f64(dev["dH"])
+    e = rel_fro(dH, ref["dH"])
+    assert e <= TOL_GRAD_FRO, f"dH rel Frobenius err {e}"
+    zero_rows = ref["coeff"] == 0
+    assert (dH[zero_rows] == 0).all(), "rows with zero coefficient must have dH == 0"
+    dW_ref = ref["dW"] if dW_before is None else ref["dW"] + dW_before
+    e = rel_fro(f64(dev["dW"]), dW_ref)
+    assert e <= TOL_GRAD_FRO, f"dW rel Frobenius err {e}"
+    return ref

@@ -1,0 +1,92 @@
+"""The shared library loads without a GPU and exports what include/drk.h declares."""
+import ctypes
+import os
+import re
+
+import pytest
+import torch
+
+from paper_2602_05885_b200 import binding as B
+from paper_2602_05885_b200 import build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build_library()
+    return B.load()
+
+
+def _declared_functions():
+    src = open(os.path.join(ROOT, "include", "drk.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(drk_[a-z0-9_]+)\s*\(", src)))
+
+
+def test_exports_every_declared_symbol(lib):
+    names = _declared_functions()
+    assert {"drk_trloo_advantage", "drk_pg_logprob_fwd", "drk_pg_loss_fwd_bwd", "drk_pg_workspace_bytes",
+            "drk_pg_params_default", "drk_status_string", "drk_version", "drk_last_launch_count"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+    # and the binding offers a function of the same name for each
+    for n in names:
+        assert hasattr(B, n), n
+
+
+def test_defaults_are_the_papers_constants():
+    p = B.drk_pg_params_default()
+    assert abs(p.mrs_lo - 0.999) < 1e-7 and abs(p.mrs_hi - 1.001) < 1e-7     # Sec. 5.1 acceptance band
+    assert abs(p.veto_ratio - 1e-4) < 1e-10                                     # Sec. 5.1 token veto
+    assert p.norm == B.DRK_NORM_KEPT_TOKENS and p.engine == B.DRK_ENGINE_AUTO
+    assert ctypes.sizeof(B.drk_pg_params) == 40
+
+
+def test_workspace_bytes():
+    p = B.drk_pg_params_default()
+    small = B.drk_pg_workspace_bytes(1024, 256, 4096, 16, B.DRK_F32, p, 1)
+    fwd = B.drk_pg_workspace_bytes(1024, 256, 4096, 16, B.DRK_F32, p, 0)
+    assert 0 < fwd < small
+    big = B.drk_pg_workspace_bytes(32768, 5120, 151936, 28, B.DRK_BF16, p, 1)
+    # bounded by the dL chunk (T x 8192 bf16) plus per-row partials: far below full logits (T x V)
+    assert big < 0.1 * 32768 * 151936 * 2
+    p.dh_dtype = B.DRK_BF16
+    assert B.drk_pg_workspace_bytes(32768, 5120, 151936, 28, B.DRK_BF16, p, 1) - big >= 32768 * 5120 * 4
+    p.v_chunk = 16384
+    assert B.drk_pg_workspace_bytes(32768, 5120, 151936, 28, B.DRK_BF16, p, 1) > big
+    # invalid arguments give 0
+    assert B.drk_pg_workspace_bytes(-1, 256, 4096, 16, B.DRK_F32, None, 1) == 0
+    assert B.drk_pg_workspace_bytes(16, 256, 0, 16, B.DRK_F32, None, 1) == 0
+    assert B.drk_pg_workspace_bytes(16, 256, 4096, 16, 5, None, 1) == 0
+    assert B.drk_pg_workspace_bytes(16, 256, 4096, 16, B.DRK_F32, None, 2) == 0
+
+
+def test_status_strings_and_version():
+    assert B.drk_version() >= 100
+    seen = {B.status_string(c) for c in range(0, -6, -1)}
+    assert len(seen) == 6 and "unknown status" not in seen
+    assert B.status_string(-99) == "unknown status"
+
+
+def test_validation_precedes_any_cuda_call():
+    # these are rejected on the host before the device is touched, so they behave the same without a GPU
+    z = torch.zeros(8)
+    assert B.drk_trloo_advantage(z, z, z, -1, 2, 1.0, 0, z, z, z, stream=0, check=False) == B.DRK_ERR_INVALID_ARG
+    assert B.drk_trloo_advantage(z, z, z, 2, 2, 1.5, 0, z, z, z, stream=0, check=False) == B.DRK_ERR_INVALID_ARG
+    assert B.drk_trloo_advantage(z, z, z, 2, 2, 1.0, 9, z, z, z, stream=0, check=False) == B.DRK_ERR_INVALID_ARG
+    assert B.drk_trloo_advantage(z, z, z, 2, 65, 1.0, 0, z, z, z, stream=0, check=False) == B.DRK_ERR_UNSUPPORTED
+    assert B.drk_trloo_advantage(None, z, z, 2, 2, 1.0, 0, z, z, z, stream=0, check=False) == B.DRK_ERR_INVALID_ARG
+    assert B.drk_pg_logprob_fwd(z, z, B.DRK_BF16, z, 8, 0, 16, 0, z, z, z, 1 << 20, z, stream=0,
+                                check=False) == B.DRK_ERR_INVALID_ARG
+    assert B.drk_last_launch_count() == 0
+
+
+@pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-GPU behaviour")
+def test_without_a_gpu_calls_fail_loudly():
+    # well-formed arguments, but no device: an error code, never a CPU fallback
+    z = torch.zeros(64)
+    rc = B.drk_trloo_advantage(z, z, z, 2, 2, 1.0, 0, z, z, z, stream=0, check=False)
+    assert rc in (B.DRK_ERR_CUDA, B.DRK_ERR_ARCH)
+    with pytest.raises(B.DrkError):
+        B.drk_trloo_advantage(z, z, z, 2, 2, 1.0, 0, z, z, z, stream=0)

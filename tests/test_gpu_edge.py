@@ -1,0 +1,108 @@
+"""Edge cases of the device path: ragged and degenerate sizes, bad inputs that only the device can see."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2602_05885_b200 import binding as B
+from tests import helpers as Hh
+from tests.gpu_utils import make_params, run_device
+
+pytestmark = pytest.mark.gpu
+
+OPEN = (0.0, math.inf, 0.0)      # MRS switched off: every sample with a masked token is retained
+
+
+@pytest.mark.parametrize("T,H,V", [(1, 64, 300), (127, 264, 4104), (129, 72, 4099), (300, 512, 257), (64, 8, 1)])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_ragged_sizes(T, H, V, dtype):
+    case = Hh.build_plain_case(f"r{T}_{H}_{V}", T=T, H=H, V=V, dtype=dtype, S=3, seed=T + V, mask_frac=0.2)
+    dev = run_device(case, make_params(*OPEN, v_chunk=256))
+    assert dev["status"] == 0
+    Hh.check_against_oracle(case, dev, *OPEN)
+
+
+def test_all_rejected_gives_exact_zero():
+    case = Hh.build_plain_case("rej", T=200, H=128, V=1000, dtype=torch.bfloat16, S=4, seed=11, sigma=0.5)
+    lo, hi, veto = float(np.float32(0.999999)), float(np.float32(1.000001)), float(np.float32(1e-4))
+    dev = run_device(case, make_params(lo, hi, veto))
+    ref = Hh.check_against_oracle(case, dev, lo, hi, veto)
+    assert ref["kept_segs"] == 0
+    assert float(dev["loss"]) == 0.0 and (dev["dH"] == 0).all() and (dev["dW"] == 0).all()
+
+
+def test_empty_inputs():
+    d = torch.device("cuda:0")
+    # S = 0: nothing to train on
+    case = Hh.build_plain_case("s0", T=130, H=64, V=500, dtype=torch.bfloat16, S=1, seed=12)
+    case.cu = torch.zeros(1, dtype=torch.int32)
+    case.seg_adv = torch.zeros(0)
+    dev = run_device(case, make_params(*OPEN))
+    assert float(dev["loss"]) == 0.0 and (dev["dH"] == 0).all() and (dev["dW"] == 0).all()
+    assert (dev["counters"] == 0).all()
+    assert np.abs(Hh.f64(dev["logp"]) - case.logp).max() <= Hh.TOL_LOGP_BF16
+    # T = 0
+    H, V = 64, 512
+    W = torch.randn(V, H).to(torch.bfloat16).to(d)
+    p = make_params(*OPEN)
+    bufs = B.PgLossBuffers(0, H, V, 2, B.DRK_BF16, p, d)
+    bufs.dW.fill_(1.0)
+    e = torch.empty(0, device=d)
+    cu = torch.zeros(3, dtype=torch.int32, device=d)
+    B.drk_pg_loss_fwd_bwd(e, W, B.DRK_BF16, e, e, e, cu, torch.ones(2, device=d), 0, H, V, 2, p, bufs.loss, bufs.logp,
+                          bufs.lse, bufs.seg_w, bufs.seg_keep, bufs.counters, bufs.dH, bufs.dW, bufs.workspace,
+                          bufs.workspace_bytes, bufs.status)
+    torch.cuda.synchronize()
+    assert float(bufs.loss.item()) == 0.0 and (bufs.dW == 0).all() and (bufs.seg_keep == 0).all()
+    assert (bufs.seg_w == 1).all()
+    assert B.drk_pg_logprob_fwd(e, W, B.DRK_BF16, e, 0, H, V, 0, e, e, bufs.workspace, bufs.workspace_bytes,
+                                bufs.status) == B.DRK_OK
+
+
+def test_device_detected_errors_set_status_bits():
+    case = Hh.build_plain_case("bad", T=140, H=64, V=700, dtype=torch.bfloat16, S=2, seed=13)
+    good = case.ids.clone()
+    case.ids[5] = 700          # outside [0, V)
+    case.ids[9] = -3
+    dev = run_device(case, make_params(*OPEN))
+    assert dev["status"] & B.DRK_STATUS_BAD_ID
+    ok = np.ones(140, dtype=bool)
+    ok[[5, 9]] = False
+    assert np.abs(Hh.f64(dev["logp"]) - case.logp)[ok].max() <= Hh.TOL_LOGP_BF16
+    # a bad row's target logit reads as 0, so logp = -lse
+    assert abs(float(dev["logp"][5]) + float(dev["lse"][5])) < 1e-6
+    case.ids = good
+    case.cu = torch.tensor([0, 90, 60], dtype=torch.int32)      # decreasing
+    dev = run_device(case, make_params(*OPEN))
+    assert dev["status"] & B.DRK_STATUS_BAD_SEGMENTS
+    assert int(dev["seg_keep"][1]) == 0
+
+
+def test_host_detected_errors_return_codes():
+    d = torch.device("cuda:0")
+    T, H, V = 64, 64, 256
+    hidden = torch.zeros((T, H), dtype=torch.bfloat16, device=d)
+    W = torch.zeros((V, H), dtype=torch.bfloat16, device=d)
+    ids = torch.zeros(T, dtype=torch.int32, device=d)
+    logp = torch.empty(T, device=d)
+    lse = torch.empty(T, device=d)
+    st = torch.zeros(1, dtype=torch.int32, device=d)
+    nb = B.drk_pg_workspace_bytes(T, H, V, 0, B.DRK_BF16, None, 0)
+    ws = torch.empty(nb, dtype=torch.uint8, device=d)
+    call = lambda **kw: B.drk_pg_logprob_fwd(kw.get("hidden", hidden), W, kw.get("dt", B.DRK_BF16), ids,
+                                             kw.get("T", T), kw.get("H", H), V, 0, logp, lse, ws,
+                                             kw.get("nb", nb), st, check=False)
+    assert call() == B.DRK_OK
+    assert call(nb=nb - 512) == B.DRK_ERR_WORKSPACE
+    assert call(T=-1) == B.DRK_ERR_INVALID_ARG
+    assert call(dt=7) == B.DRK_ERR_INVALID_ARG
+    assert call(H=68) == B.DRK_ERR_UNSUPPORTED            # bf16 rows must be 16-byte multiples
+    assert call(hidden=hidden.view(-1)[1:]) == B.DRK_ERR_INVALID_ARG   # misaligned
+    assert B.drk_last_launch_count() == 0
+    torch.cuda.synchronize()
+    # W = 0: uniform distribution, logp = -ln V exactly up to rounding
+    assert call() == B.DRK_OK
+    torch.cuda.synchronize()
+    assert torch.allclose(logp, torch.full_like(logp, -math.log(V)), atol=1e-5)
+    assert B.drk_last_launch_count() == 2

@@ -1,0 +1,120 @@
+"""Device path against the oracle, element by element, on the tiny config and on reduced-T versions of
+the 8B-, 14B- and ragged-shaped configs (same H, V, dtype and structure; T spans several row tiles and
+ends in a ragged one)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2602_05885_b200 import binding as B
+from tests import helpers as Hh
+from tests.gpu_utils import make_params, run_device
+
+pytestmark = pytest.mark.gpu
+
+F32 = lambda x: float(np.float32(x))
+PAPER = (F32(0.999), F32(1.001), F32(1e-4))
+
+
+def _case_tiny(seed):
+    # 2 prompts x 4 rollouts x 2 turns x 64 response tokens, fp32
+    return Hh.build_case(f"tiny{seed}", H=256, V=4096, dtype=torch.float32, P=2, K=4, Tmax=2, len_lo=64, len_hi=64,
+                         capacity=1024, seed=seed, sigma=0.05)
+
+
+CASES = {
+    "tiny0": lambda: _case_tiny(0),
+    "tiny1": lambda: _case_tiny(1),
+    "tiny2": lambda: _case_tiny(2),
+    # 8B-shaped: lengths scaled down 8x so that a 700-token micro-batch holds whole segments
+    "q8b": lambda: Hh.build_case("q8b", H=4096, V=151936, dtype=torch.bfloat16, P=16, K=8, Tmax=3, len_lo=16,
+                                 len_hi=128, capacity=700, seed=1000, sigma=0.05),
+    # 14B-shaped: mismatch noise 0.1, 1 % outliers concentrated in 10 % of the segments
+    "q14b": lambda: Hh.build_case("q14b", H=5120, V=151936, dtype=torch.bfloat16, P=32, K=8, Tmax=3, len_lo=32,
+                                  len_hi=256, capacity=650, seed=2000, sigma=0.1, outlier_frac=0.01),
+    # ragged multi-turn: 4 turns, early termination, 40 % unmasked context, padding in front and behind
+    "ragged": lambda: Hh.build_case("ragged", H=5120, V=151936, dtype=torch.bfloat16, P=32, K=8, Tmax=4, len_lo=16,
+                                    len_hi=96, capacity=600, seed=3000, sigma=0.1, outlier_frac=0.01, ragged=True,
+                                    ctx_frac=0.4, lead_pad=5),
+    # several waves of work units per SM and several vocabulary chunks
+    "medium": lambda: Hh.build_case("medium", H=1024, V=8200, dtype=torch.bfloat16, P=16, K=8, Tmax=3, len_lo=64,
+                                    len_hi=512, capacity=5000, seed=4000, sigma=0.05),
+}
+_cache = {}
+
+
+def get_case(name):
+    if name not in _cache:
+        if len(_cache) >= 2:            # the big cases hold GBs of oracle logits
+            _cache.pop(next(iter(_cache)))
+        _cache[name] = CASES[name]()
+    return _cache[name]
+
+
+@pytest.mark.parametrize("name", ["tiny0", "tiny1", "tiny2"])
+def test_tiny_fp32(name):
+    case = get_case(name)
+    for (lo, hi, veto) in (PAPER, Hh.wide_band(case) + (PAPER[2],), (0.0, math.inf, 0.0)):
+        dev = run_device(case, make_params(lo, hi, veto))
+        assert dev["status"] == 0
+        Hh.check_against_oracle(case, dev, lo, hi, veto)
+
+
+def test_tiny_forward_only_and_determinism():
+    case = get_case("tiny0")
+    d = torch.device("cuda:0")
+    a = B.pg_logprob_fwd(case.hidden.to(d), case.W.to(d), case.ids.to(d))
+    b = B.pg_logprob_fwd(case.hidden.to(d), case.W.to(d), case.ids.to(d))
+    torch.cuda.synchronize()
+    assert np.abs(Hh.f64(a[0]) - case.logp).max() <= Hh.TOL_LOGP_F32
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    assert int(a[2].item()) == 0
+
+
+@pytest.mark.parametrize("name", ["medium", "q8b", "q14b", "ragged"])
+@pytest.mark.parametrize("engine", [B.DRK_ENGINE_AUTO, B.DRK_ENGINE_SIMT])
+def test_bf16_shapes(name, engine):
+    if engine == B.DRK_ENGINE_SIMT and name in ("q14b", "ragged"):
+        pytest.skip("FFMA cross-check runs on two bf16 shapes only (time)")
+    case = get_case(name)
+    wide = Hh.wide_band(case)
+    for (lo, hi, veto) in (PAPER, wide + (PAPER[2],)):
+        dev = run_device(case, make_params(lo, hi, veto, engine=engine, v_chunk=2048 if name == "medium" else 0))
+        assert dev["status"] == 0
+        ref = Hh.check_against_oracle(case, dev, lo, hi, veto)
+        if (lo, hi) == wide:
+            assert 0 < ref["kept_segs"] < case.S        # both retained and rejected samples present
+
+
+def test_bf16_output_dtypes_accumulate_and_norms():
+    case = get_case("medium")
+    lo, hi = Hh.wide_band(case)
+    veto = PAPER[2]
+    # bf16 gradients
+    dev = run_device(case, make_params(lo, hi, veto, dw_dtype=B.DRK_BF16, dh_dtype=B.DRK_BF16, v_chunk=4096))
+    Hh.check_against_oracle(case, dev, lo, hi, veto)
+    # dW accumulation on top of existing values, fp32 and bf16
+    g = torch.Generator().manual_seed(5)
+    init = (torch.randn((case.V, case.H), generator=g) * 1e-4)
+    for dt, tdt in ((B.DRK_F32, torch.float32), (B.DRK_BF16, torch.bfloat16)):
+        init_t = init.to(tdt)
+        dev = run_device(case, make_params(lo, hi, veto, dw_dtype=dt, dw_accumulate=1), dW_init=init_t)
+        Hh.check_against_oracle(case, dev, lo, hi, veto, dW_before=Hh.f64(init_t))
+    # other normalisations
+    dev = run_device(case, make_params(lo, hi, veto, norm=B.DRK_NORM_ALL_MASKED_TOKENS))
+    Hh.check_against_oracle(case, dev, lo, hi, veto, norm=1)
+    dev = run_device(case, make_params(lo, hi, veto, norm=B.DRK_NORM_EXPLICIT, explicit_scale=F32(1 / 4096)))
+    Hh.check_against_oracle(case, dev, lo, hi, veto, norm=2, explicit_scale=F32(1 / 4096))
+
+
+def test_end_to_end_with_device_advantages():
+    # advantages from drk_trloo_advantage feed the device loss; the oracle uses its own
+    case = get_case("q8b")
+    d = torch.device("cuda:0")
+    rb = case.rb
+    _, adv, _ = B.trloo_advantage(rb.reward.to(d), rb.valid.to(d), rb.prompt_of_rollout.to(d))
+    seg_adv_dev = adv[case.seg_rollout.to(d), case.seg_turn.to(d)].contiguous().cpu()
+    lo, hi = Hh.wide_band(case)
+    dev = run_device(case, make_params(lo, hi, PAPER[2]), seg_adv=seg_adv_dev)
+    Hh.check_against_oracle(case, dev, lo, hi, PAPER[2])
