@@ -1,0 +1,61 @@
+"""The data-parallel host logic on two gloo ranks (CPU): disjoint micro-batch ownership and the
+max-over-ranks time that defines whole-job throughput."""
+import os
+import socket
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from paper_2602_05885_b200 import dp, synth
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def _worker(rank, world, port, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    rb = synth.rollout_batch(4, 8, 3, 16, 128, seed=11)
+    plans = synth.pack_first_fit(rb, 700)
+    owned = dp.assign_microbatches([p.used for p in plans], world)
+    mine = owned[rank]
+    tokens = sum(plans[i].used for i in mine)
+    t_rank = 1.0 + rank            # pretend rank 1 is slower
+    t_job = dp.max_over_ranks(t_rank)
+    total = dp.sum_over_ranks(tokens)
+    out.put((rank, mine, tokens, t_job, total, len(plans), sum(p.used for p in plans)))
+    dist.destroy_process_group()
+
+
+def test_two_rank_sharding_and_timing():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    (_, a, ta, ja, tot_a, n, all_tokens), (_, b, tb, jb, tot_b, _, _) = res
+    assert sorted(a + b) == list(range(n)) and not set(a) & set(b)     # every micro-batch exactly once
+    assert ja == jb == 2.0                                             # job time = slowest rank
+    assert tot_a == tot_b == all_tokens == ta + tb
+    assert abs(ta - tb) <= 700                                         # balanced within one micro-batch
+
+
+def test_assignment_balances_and_covers():
+    loads = [700, 10, 650, 640, 30, 500, 20]
+    owned = dp.assign_microbatches(loads, 3)
+    assert sorted(i for o in owned for i in o) == list(range(7))
+    tot = [sum(loads[i] for i in o) for o in owned]
+    assert max(tot) - min(tot) <= 700
+    assert dp.max_over_ranks(3.5) == 3.5 and dp.sum_over_ranks(2.0) == 2.0   # no process group: identity

@@ -1,0 +1,165 @@
+"""Parity at the benchmark's full size (T=32768, H=5120, V=151936, bf16) and launch configuration.
+
+The full fp64 oracle would need ~1.5e14 flops here, so two routes are used:
+
+  * structured inputs: the hidden rows are drawn from 48 distinct rows (the device path neither knows nor
+    cares).  Rows that are exact copies have exactly the same logits, so the oracle evaluates every token's
+    log-prob from the 48 distinct logit rows, block by block, with its ordinary functions; MRS, coefficients
+    and the loss follow for all T.  dH is checked on a sample of rows (each row of dH depends on its own token
+    only).  dW is linear in the per-token dLogits: tokens sharing a hidden row share their softmax term, so
+    the oracle's dW of the 48-row problem with summed coefficients, corrected by the (sparse) one-hot terms,
+    equals the full dW; every element is compared.
+  * the benchmark's own inputs: sampled rows (log-prob, lse, dH) plus the identity sum_v dW[v,:] = 0.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import drk_oracle as O
+from paper_2602_05885_b200 import binding as B
+from paper_2602_05885_b200 import workload
+from tests import helpers as Hh
+
+pytestmark = pytest.mark.gpu
+
+F32 = lambda x: float(np.float32(x))
+
+
+def _bench_params(wl, mrs="wide"):
+    p = B.drk_pg_params_default()
+    if mrs == "wide":
+        lo, hi = wl.wide_band()
+        p.mrs_lo, p.mrs_hi = lo, hi
+    else:
+        p.mrs_lo, p.mrs_hi, p.veto_ratio = 0.0, float("inf"), 0.0
+    p.dw_dtype = B.DRK_F32
+    p.dh_dtype = B.DRK_BF16
+    return p
+
+
+def _run(wl, p, seg_adv):
+    dev = wl.hidden.device
+    bufs = B.PgLossBuffers(wl.T, wl.H, wl.V, wl.S, B.DRK_BF16, p, dev)
+    B.drk_pg_loss_fwd_bwd(wl.hidden, wl.W, B.DRK_BF16, wl.ids, wl.rollout_logp, wl.loss_mask, wl.cu, seg_adv,
+                          wl.T, wl.H, wl.V, wl.S, p, bufs.loss, bufs.logp, bufs.lse, bufs.seg_w, bufs.seg_keep,
+                          bufs.counters, bufs.dH, bufs.dW, bufs.workspace, bufs.workspace_bytes, bufs.status)
+    torch.cuda.synchronize()
+    assert int(bufs.status.item()) == 0
+    return bufs
+
+
+def test_full_size_structured_rows():
+    dev = torch.device("cuda:0")
+    R = 48
+    wl = workload.build("qwen3-14b", dev, seed=2100, distinct_rows=R)
+    T, H, V, S = wl.T, wl.H, wl.V, wl.S
+    assert (T, H, V) == (32768, 5120, 151936)
+    g = torch.Generator().manual_seed(7)
+    seg_adv = torch.randn(S, generator=g).float()
+    p = _bench_params(wl)
+    bufs = _run(wl, p, seg_adv.to(dev))
+
+    # ---- oracle side: inputs only
+    row_of = wl.row_of.cpu().numpy()
+    hidden_cpu = wl.hidden.cpu()
+    # one representative token per distinct row
+    first = np.full(R, -1, dtype=np.int64)
+    for t in range(T - 1, -1, -1):
+        first[row_of[t]] = t
+    used = first >= 0
+    base = Hh.f64(hidden_cpu[torch.from_numpy(first[used])])
+    remap = np.cumsum(used) - 1
+    row_idx = remap[row_of]
+    W64 = Hh.f64(wl.W.cpu())
+    ids = wl.ids.cpu().numpy().astype(np.int64)
+    s_r = O.logits(base, W64)                                   # [R', V]
+    logp = np.empty(T)
+    lse = np.empty(T)
+    for a in range(0, T, 2048):
+        b = min(T, a + 2048)
+        logp[a:b], lse[a:b] = O.token_logprob(s_r[row_idx[a:b]], ids[a:b])
+    assert np.abs(Hh.f64(bufs.logp) - logp).max() <= Hh.TOL_LOGP_BF16
+    assert np.abs(Hh.f64(bufs.lse) - lse).max() <= Hh.TOL_LOGP_BF16
+
+    lo, hi, veto = float(p.mrs_lo), float(p.mrs_hi), float(p.veto_ratio)
+    rl = Hh.f64(wl.rollout_logp)
+    mask = wl.loss_mask.cpu().numpy()
+    cu = wl.cu.cpu().numpy()
+    m = O.mrs(logp, rl, mask, cu, lo, hi, veto)
+    keep_dev = bufs.seg_keep.cpu().numpy().astype(bool)
+    amb = Hh.ambiguous_segments(m, lo, hi, veto, Hh.TOL_LOGP_BF16, Hh.TOL_LOGP_BF16)
+    assert not ((keep_dev != m.keep) & ~amb).any()
+    lr = O.coeff_and_loss(logp, keep_dev, mask, cu, Hh.f64(seg_adv))
+    cnt = bufs.counters.cpu().numpy()
+    assert cnt[0] == lr.kept_tokens and cnt[1] == lr.masked_tokens and cnt[2] == lr.kept_segs
+    assert 0 < lr.kept_segs < S
+    denom = max(abs(lr.loss), 1e-3 * float(np.sum(np.abs(lr.coeff * logp))))
+    assert abs(float(bufs.loss.item()) - lr.loss) / denom <= Hh.TOL_LOSS_REL
+
+    # ---- dH on sampled rows (incl. rows with zero coefficient)
+    rng = np.random.default_rng(3)
+    sample = np.sort(rng.choice(T, size=384, replace=False))
+    s_s = s_r[row_idx[sample]]
+    dH_s, _ = O.gradients(Hh.f64(hidden_cpu[torch.from_numpy(sample)]), W64, s_s, lse[sample], ids[sample],
+                          lr.coeff[sample])
+    dH_dev = Hh.f64(bufs.dH[torch.from_numpy(sample).to(dev)])
+    assert Hh.rel_fro(dH_dev, dH_s) <= Hh.TOL_GRAD_FRO
+    zero = lr.coeff == 0
+    assert zero.any() and (~zero).any()
+    assert float(bufs.dH[torch.from_numpy(np.nonzero(zero)[0]).to(dev)].abs().max()) == 0.0
+    del s_s, dH_s
+
+    # ---- dW, every element: 48-row problem with summed coefficients + one-hot corrections
+    Rn = base.shape[0]
+    csum = np.zeros(Rn)
+    np.add.at(csum, row_idx, lr.coeff)
+    lse_r = O.logsumexp_rows(s_r)
+    _, dW = O.gradients(base, W64, s_r, lse_r, np.zeros(Rn, dtype=np.int64), csum)
+    dW[0] += csum @ base                                        # undo the reduced problem's one-hot at id 0
+    nz = np.nonzero(lr.coeff)[0]
+    np.subtract.at(dW, ids[nz], lr.coeff[nz, None] * base[row_idx[nz]])
+    dW_dev = bufs.dW.cpu()
+    num = 0.0
+    for a in range(0, V, 8192):                                  # blockwise to bound memory
+        blk = Hh.f64(dW_dev[a:a + 8192]) - dW[a:a + 8192]
+        num += float(np.sum(blk * blk))
+    err = math.sqrt(num) / float(np.linalg.norm(dW))
+    assert err <= Hh.TOL_GRAD_FRO, f"dW rel Frobenius err {err}"
+
+
+def test_full_size_bench_inputs_sampled_rows():
+    dev = torch.device("cuda:0")
+    wl = workload.build("qwen3-14b", dev, seed=2000)
+    T, H, V, S = wl.T, wl.H, wl.V, wl.S
+    # MRS off and an explicit scale: every coefficient is then known without the other rows' log-probs
+    p = _bench_params(wl, mrs="off")
+    p.norm = B.DRK_NORM_EXPLICIT
+    p.explicit_scale = F32(1.0 / 32768)
+    g = torch.Generator().manual_seed(8)
+    seg_adv = torch.randn(S, generator=g).float()
+    bufs = _run(wl, p, seg_adv.to(dev))
+    mask = wl.loss_mask.cpu().numpy()
+    cu = wl.cu.cpu().numpy()
+    keep = np.array([mask[cu[j]:cu[j + 1]].any() for j in range(S)])
+    assert np.array_equal(bufs.seg_keep.cpu().numpy().astype(bool), keep)
+    lr = O.coeff_and_loss(np.zeros(T), keep, mask, cu, Hh.f64(seg_adv), O.NORM_EXPLICIT, float(p.explicit_scale))
+    rng = np.random.default_rng(4)
+    sample = np.sort(rng.choice(T, size=256, replace=False))
+    st = torch.from_numpy(sample)
+    hid = Hh.f64(wl.hidden[st.to(dev)])
+    W64 = Hh.f64(wl.W.cpu())
+    ids = wl.ids.cpu().numpy().astype(np.int64)[sample]
+    s = O.logits(hid, W64)
+    logp, lse = O.token_logprob(s, ids)
+    assert np.abs(Hh.f64(bufs.logp)[sample] - logp).max() <= Hh.TOL_LOGP_BF16
+    assert np.abs(Hh.f64(bufs.lse)[sample] - lse).max() <= Hh.TOL_LOGP_BF16
+    dH_s, _ = O.gradients(hid, W64, s, lse, ids, lr.coeff[sample])
+    assert Hh.rel_fro(Hh.f64(bufs.dH[st.to(dev)]), dH_s) <= Hh.TOL_GRAD_FRO
+    # every row of softmax - onehot sums to zero, hence so do the columns of dW over the vocabulary
+    dW = bufs.dW
+    colsum = dW.double().sum(dim=0)
+    scale = dW.double().abs().sum(dim=0)
+    assert float((colsum.abs() / scale.clamp(min=1e-30)).max()) < 2e-3
+    assert float(dW.abs().max()) > 0
