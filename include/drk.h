@@ -124,6 +124,29 @@ int drk_pg_logprob_fwd(const void* hidden, const void* W, int32_t in_dtype, cons
                        void* workspace, size_t workspace_bytes, uint32_t* status, void* stream);
 
 /*
+ * The same computation as drk_pg_logprob_fwd for callers that cannot hand over a workspace because they
+ * cannot allocate device memory when the call is made: for instance a training loop whose framework
+ * already owns all of HBM through its own pool, or a latency-critical section that must avoid
+ * cudaMalloc's implicit synchronisation.  (The paper has no counterpart for this entry point; it is a
+ * packaging variant of the forward call above.)  The scratch (per-row partial max / sum-exp pairs and
+ * target logits) lives in a fixed array inside the library image instead:
+ *   - every GPU on which the library is loaded holds DRK_NOALLOC_SCRATCH_BYTES until the process exits;
+ *   - if the sizes need more (roughly 8*nsplit*T + 4*T bytes, nsplit <= 32 chosen from T and V) the call
+ *     returns DRK_ERR_WORKSPACE and enqueues nothing; T = 32768 at V = 151936 needs about 1.2 MB;
+ *   - the array is shared by all calls on a device and keeps the last call's contents.  What the
+ *     computation reads is rewritten or cleared by each call, so consecutive calls on one stream are
+ *     independent; calls that may run concurrently on the GPU (unordered streams) race on it;
+ *   - the first call on each device looks up the array's device address.  Make that first call
+ *     outside any stream capture.
+ * It calls no cudaMalloc / cudaFree and no allocating library routine.  Arguments, outputs, status bits
+ * and return codes are those of drk_pg_logprob_fwd, without the workspace pair.
+ */
+#define DRK_NOALLOC_SCRATCH_BYTES (8u << 20)
+int drk_pg_logprob_fwd_noalloc(const void* hidden, const void* W, int32_t in_dtype, const int32_t* ids,
+                               int64_t T, int32_t H, int32_t V, int32_t engine, float* logp, float* lse,
+                               uint32_t* status, void* stream);
+
+/*
  * Loss and gradients of one packed micro-batch: forward as above, geometric
  * mismatch rejection sampling with token veto per training sample (Sec. 5.1),
  * the REINFORCE surrogate with the caller's per-sample advantages (App. A,

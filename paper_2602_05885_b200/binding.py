@@ -86,6 +86,8 @@ def load() -> ctypes.CDLL:
     lib.drk_trloo_advantage.restype = ctypes.c_int
     lib.drk_pg_logprob_fwd.argtypes = [vp, vp, i32, vp, i64, i32, i32, i32, vp, vp, vp, sz, vp, vp]
     lib.drk_pg_logprob_fwd.restype = ctypes.c_int
+    lib.drk_pg_logprob_fwd_noalloc.argtypes = [vp, vp, i32, vp, i64, i32, i32, i32, vp, vp, vp, vp]
+    lib.drk_pg_logprob_fwd_noalloc.restype = ctypes.c_int
     lib.drk_pg_loss_fwd_bwd.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, i64, i32, i32, i32,
                                         ctypes.POINTER(drk_pg_params), vp, vp, vp, vp, vp, vp, vp, vp, vp, sz,
                                         vp, vp]
@@ -163,6 +165,22 @@ def drk_pg_logprob_fwd(hidden, W, in_dtype: int, ids, T: int, H: int, V: int, en
                                    _ptr(workspace), workspace_bytes, _ptr(status), _stream(stream))
     if check and rc != DRK_OK:
         raise DrkError(rc, "drk_pg_logprob_fwd")
+    return rc
+
+
+DRK_NOALLOC_SCRATCH_BYTES = 8 << 20
+
+
+def drk_pg_logprob_fwd_noalloc(hidden, W, in_dtype: int, ids, T: int, H: int, V: int, engine: int, logp, lse,
+                               status, stream=None, check: bool = True) -> int:
+    """drk_pg_logprob_fwd without a workspace argument: the scratch is a fixed array inside libdrk.so
+    (DRK_NOALLOC_SCRATCH_BYTES per GPU), for callers that cannot allocate device memory at call time.
+    Sizes that need more return DRK_ERR_WORKSPACE.  Calls on one device share the array: keep them on one
+    stream or otherwise ordered.  Make the first call on a device outside any stream capture."""
+    rc = load().drk_pg_logprob_fwd_noalloc(_ptr(hidden), _ptr(W), in_dtype, _ptr(ids), T, H, V, engine, _ptr(logp),
+                                           _ptr(lse), _ptr(status), _stream(stream))
+    if check and rc != DRK_OK:
+        raise DrkError(rc, "drk_pg_logprob_fwd_noalloc")
     return rc
 
 
