@@ -47,8 +47,10 @@ typedef enum {
   DRK_NORM_EXPLICIT = 2           /* scale = explicit_scale                                      */
 } drk_norm;
 typedef enum {
-  DRK_ENGINE_AUTO = 0, /* bf16 inputs: tcgen05 tensor-core kernels; fp32 inputs: fp32 FFMA kernels */
-  DRK_ENGINE_SIMT = 1  /* force the FFMA kernels (exact fp32 products; slow; for cross-checks)     */
+  DRK_ENGINE_AUTO = 0,     /* bf16 inputs: tcgen05 tensor-core kernels on CTA pairs (256x256 tiles);
+                              fp32 inputs: fp32 FFMA kernels                                        */
+  DRK_ENGINE_SIMT = 1,     /* force the FFMA kernels (exact fp32 products; slow; for cross-checks)  */
+  DRK_ENGINE_UMMA_1CTA = 2 /* bf16 inputs: tcgen05 kernels with one CTA per 128x256 tile           */
 } drk_engine;
 
 /* Bits of the device status word. */

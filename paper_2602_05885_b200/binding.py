@@ -31,6 +31,7 @@ DRK_NORM_ALL_MASKED_TOKENS = 1
 DRK_NORM_EXPLICIT = 2
 DRK_ENGINE_AUTO = 0
 DRK_ENGINE_SIMT = 1
+DRK_ENGINE_UMMA_1CTA = 2
 
 DRK_STATUS_BAD_ID = 1
 DRK_STATUS_BAD_SEGMENTS = 2

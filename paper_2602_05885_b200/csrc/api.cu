@@ -21,6 +21,8 @@ int check_arch() {
 }
 
 bool use_simt(int in_dtype, int engine) { return in_dtype == DRK_F32 || engine == DRK_ENGINE_SIMT; }
+int umma_ctas(int engine) { return engine == DRK_ENGINE_UMMA_1CTA ? 1 : 2; }
+bool engine_ok(int e) { return e == DRK_ENGINE_AUTO || e == DRK_ENGINE_SIMT || e == DRK_ENGINE_UMMA_1CTA; }
 
 bool sizes_ok(int64_t T, int H, int V, int in_dtype) {
   if (T < 0 || T > (1 << 24) || H < 1 || H > 65536 || V < 1 || V > (1 << 24)) return false;
@@ -28,8 +30,35 @@ bool sizes_ok(int64_t T, int H, int V, int in_dtype) {
   return true;
 }
 
-int round_vchunk(int v_chunk, int V) {
-  int vc = v_chunk > 0 ? v_chunk : kDefaultVChunk;
+// Chunk width for the tensor-core backward when the caller leaves it to the library: the multiple of
+// 256 that minimises the modelled time of the three per-chunk kernels.  Each kernel is persistent
+// over 148 SMs with 128x256 tiles, so its time is (waves of tiles) x (k-blocks per tile); a fixed
+// cost per launch stands for fill and drain.  The dL buffer is kept below ~1 GiB.
+int auto_vchunk(int64_t T, int H, int V) {
+  const int64_t sms = 148, launch_cost = 96;
+  const int64_t mt_T = ceil_div(T, 128), nt_H = ceil_div(H, 256), kb_H = ceil_div(H, 64), kb_T = ceil_div(T, 64);
+  int64_t cap = ((int64_t)1 << 30) / (2 * (T > 0 ? T : 1)) / 256 * 256;
+  if (cap < 8192) cap = 8192;
+  if (cap > 32768) cap = 32768;
+  const int64_t vmax = ceil_div(V, 256) * 256;
+  int best = 0;
+  double best_cost = 0;
+  for (int64_t vc = 2048; vc <= cap; vc += 256) {
+    double cost = 0;
+    for (int64_t v0 = 0; v0 < V; v0 += vc) {
+      const int64_t w = V - v0 < vc ? V - v0 : vc;
+      cost += (double)(ceil_div(mt_T * ceil_div(w, 256), sms) * kb_H + launch_cost);   // DL
+      cost += (double)(ceil_div(ceil_div(w, 128) * nt_H, sms) * kb_T + launch_cost);   // DW
+      cost += (double)(ceil_div(mt_T * nt_H, sms) * ceil_div(w, 64) + launch_cost);    // DH
+    }
+    if (best == 0 || cost < best_cost) { best = (int)vc; best_cost = cost; }
+    if (vc >= vmax) break;
+  }
+  return best;
+}
+
+int round_vchunk(int v_chunk, int64_t T, int H, int V, bool simt) {
+  int vc = v_chunk > 0 ? v_chunk : (simt ? kDefaultVChunk : auto_vchunk(T, H, V));
   vc = (int)(ceil_div(vc, 256) * 256);
   const int vmax = (int)(ceil_div(V, 256) * 256);
   return vc < vmax ? vc : vmax;
@@ -52,9 +81,9 @@ struct FwdWs {
   float* tgt;
   int nsplit;
 };
-FwdWs carve_fwd(Carver& c, int64_t T, int V, bool simt) {
+FwdWs carve_fwd(Carver& c, int64_t T, int V, bool simt, int engine) {
   FwdWs w;
-  w.nsplit = simt ? simt_nsplit(T, V) : umma_nsplit(T, V);
+  w.nsplit = simt ? simt_nsplit(T, V) : umma_nsplit(T, V, umma_ctas(engine));
   w.part = static_cast<float*>(c.take(sizeof(float) * 2 * (size_t)w.nsplit * (size_t)T));
   w.tgt = static_cast<float*>(c.take(sizeof(float) * (size_t)T));
   return w;
@@ -69,7 +98,7 @@ struct BwdWs {
 };
 BwdWs carve_bwd(Carver& c, int64_t T, int H, int V, int S, bool simt, const drk_pg_params& p) {
   BwdWs w;
-  w.vc = round_vchunk(p.v_chunk, V);
+  w.vc = round_vchunk(p.v_chunk, T, H, V, simt);
   w.coeff = static_cast<float*>(c.take(sizeof(float) * (size_t)T));
   w.seg_stats = static_cast<double*>(c.take(sizeof(double) * 4 * (size_t)S));
   w.dL = c.take((simt ? 4 : 2) * (size_t)T * (size_t)w.vc);
@@ -81,7 +110,7 @@ bool params_ok(const drk_pg_params& p) {
   if (p.norm < 0 || p.norm > 2) return false;
   if (p.dw_dtype != DRK_F32 && p.dw_dtype != DRK_BF16) return false;
   if (p.dh_dtype != DRK_F32 && p.dh_dtype != DRK_BF16) return false;
-  if (p.engine != DRK_ENGINE_AUTO && p.engine != DRK_ENGINE_SIMT) return false;
+  if (!engine_ok(p.engine)) return false;
   if (p.v_chunk < 0) return false;
   if (std::isnan(p.mrs_lo) || std::isnan(p.mrs_hi) || std::isnan(p.veto_ratio)) return false;
   if (p.norm == DRK_NORM_EXPLICIT && !std::isfinite(p.explicit_scale)) return false;
@@ -89,12 +118,12 @@ bool params_ok(const drk_pg_params& p) {
 }
 
 int run_fwd(const void* hidden, const void* W, int in_dtype, const int32_t* ids, int64_t T, int H, int V,
-            bool simt, const FwdWs& w, float* logp, float* lse, uint32_t* status, cudaStream_t st) {
+            bool simt, int engine, const FwdWs& w, float* logp, float* lse, uint32_t* status, cudaStream_t st) {
   if (simt) {
     SimtFwdArgs a{hidden, W, in_dtype, ids, T, H, V, logp, lse, w.part, w.tgt, w.nsplit, status};
     return launch_simt_fwd(a, st);
   }
-  UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, w.part, w.tgt, w.nsplit, status};
+  UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, w.part, w.tgt, w.nsplit, status, umma_ctas(engine)};
   return launch_umma_fwd(a, st);
 }
 
@@ -126,7 +155,7 @@ size_t drk_pg_workspace_bytes(int64_t T, int32_t H, int32_t V, int32_t S, int32_
   if (!sizes_ok(T, H, V, in_dtype) || S < 0 || !params_ok(p) || (which != 0 && which != 1)) return 0;
   const bool simt = use_simt(in_dtype, p.engine);
   Carver c(nullptr);
-  carve_fwd(c, T, V, simt);
+  carve_fwd(c, T, V, simt, p.engine);
   if (which == 1) carve_bwd(c, T, H, V, S, simt, p);
   return c.off + 256;  // never 0 for valid arguments
 }
@@ -154,7 +183,7 @@ int drk_pg_logprob_fwd(const void* hidden, const void* W, int32_t in_dtype, cons
                        size_t workspace_bytes, uint32_t* status, void* stream) {
   g_launches = 0;
   if (!sizes_ok(T, H, V, in_dtype)) return DRK_ERR_INVALID_ARG;
-  if (engine != DRK_ENGINE_AUTO && engine != DRK_ENGINE_SIMT) return DRK_ERR_INVALID_ARG;
+  if (!engine_ok(engine)) return DRK_ERR_INVALID_ARG;
   if (T == 0) return DRK_OK;
   if (!hidden || !W || !ids || !logp || !lse || !workspace || !status) return DRK_ERR_INVALID_ARG;
   if (!aligned(hidden, 16) || !aligned(W, 16) || !aligned(workspace, 256)) return DRK_ERR_INVALID_ARG;
@@ -167,8 +196,8 @@ int drk_pg_logprob_fwd(const void* hidden, const void* W, int32_t in_dtype, cons
   int rc = check_arch();
   if (rc != DRK_OK) return rc;
   Carver c(workspace);
-  const FwdWs w = carve_fwd(c, T, V, simt);
-  rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, w, logp, lse, status, static_cast<cudaStream_t>(stream));
+  const FwdWs w = carve_fwd(c, T, V, simt, engine);
+  rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, engine, w, logp, lse, status, static_cast<cudaStream_t>(stream));
   if (rc != DRK_OK) g_launches = 0;
   return rc;
 }
@@ -197,13 +226,13 @@ int drk_pg_loss_fwd_bwd(const void* hidden, const void* W, int32_t in_dtype, con
   cudaStream_t st = static_cast<cudaStream_t>(stream);
 
   Carver c(workspace);
-  const FwdWs fw = carve_fwd(c, T, V, simt);
+  const FwdWs fw = carve_fwd(c, T, V, simt, p.engine);
   const BwdWs bw = carve_bwd(c, T, H, V, S, simt, p);
 
   auto fail = [&](int code) { g_launches = 0; return code; };
 
   if (T > 0) {
-    rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, fw, logp, lse, status, st);
+    rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, p.engine, fw, logp, lse, status, st);
     if (rc != DRK_OK) return fail(rc);
   }
   MrsArgs m{};
@@ -232,7 +261,7 @@ int drk_pg_loss_fwd_bwd(const void* hidden, const void* W, int32_t in_dtype, con
     rc = launch_simt_bwd(b, st);
   } else {
     UmmaBwdArgs b{hidden, W, ids, T, H, V, lse, bw.coeff, static_cast<__nv_bfloat16*>(bw.dL), bw.vc,
-                  dH, p.dh_dtype, bw.dH_acc, dW, p.dw_dtype, p.dw_accumulate, status};
+                  dH, p.dh_dtype, bw.dH_acc, dW, p.dw_dtype, p.dw_accumulate, status, umma_ctas(p.engine)};
     rc = launch_umma_bwd(b, st);
   }
   if (rc != DRK_OK) return fail(rc);

@@ -67,13 +67,15 @@ int launch_simt_bwd(const SimtBwdArgs& a, cudaStream_t st);
 struct UmmaFwdArgs {
   const void* hidden; const void* W; const int32_t* ids; int64_t T; int H; int V;
   float* logp; float* lse; float* part /*[nsplit*T*2]*/; float* tgt; int nsplit; uint32_t* status;
+  int ctas /*1: one CTA per tile; 2: CTA pairs*/;
 };
-int umma_nsplit(int64_t T, int V);
+int umma_nsplit(int64_t T, int V, int ctas);
 int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st);
 struct UmmaBwdArgs {
   const void* hidden; const void* W; const int32_t* ids; int64_t T; int H; int V;
   const float* lse; const float* coeff; __nv_bfloat16* dL /*[T*vc]*/; int vc;
   void* dH; int dh_dtype; float* dH_acc; void* dW; int dw_dtype; int dw_accumulate; uint32_t* status;
+  int ctas;
 };
 int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st);
 

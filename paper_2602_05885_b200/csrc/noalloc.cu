@@ -63,7 +63,7 @@ extern "C" int drk_pg_logprob_fwd_noalloc(const void* hidden, const void* W, int
   g_launches = 0;
   if (T < 0 || T > (1 << 24) || H < 1 || H > 65536 || V < 1 || V > (1 << 24)) return DRK_ERR_INVALID_ARG;
   if (in_dtype != DRK_F32 && in_dtype != DRK_BF16) return DRK_ERR_INVALID_ARG;
-  if (engine != DRK_ENGINE_AUTO && engine != DRK_ENGINE_SIMT) return DRK_ERR_INVALID_ARG;
+  if (engine != DRK_ENGINE_AUTO && engine != DRK_ENGINE_SIMT && engine != DRK_ENGINE_UMMA_1CTA) return DRK_ERR_INVALID_ARG;
   if (T == 0) return DRK_OK;
   if (!hidden || !W || !ids || !logp || !lse || !status) return DRK_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(hidden) % 16 || reinterpret_cast<uintptr_t>(W) % 16) return DRK_ERR_INVALID_ARG;
@@ -71,7 +71,8 @@ extern "C" int drk_pg_logprob_fwd_noalloc(const void* hidden, const void* W, int
   if (!simt && (H % 8) != 0) return DRK_ERR_UNSUPPORTED;
 
   // scratch layout: partials [nsplit, T, 2] floats, then target logits [T] floats, each 256-aligned
-  const int nsplit = simt ? simt_nsplit(T, V) : umma_nsplit(T, V);
+  const int ctas = engine == DRK_ENGINE_UMMA_1CTA ? 1 : 2;
+  const int nsplit = simt ? simt_nsplit(T, V) : umma_nsplit(T, V, ctas);
   const size_t part_bytes = align_up(sizeof(float) * 2 * (size_t)nsplit * (size_t)T, 256);
   const size_t tgt_bytes = align_up(sizeof(float) * (size_t)T, 256);
   if (part_bytes + tgt_bytes > kScratchBytes) return DRK_ERR_WORKSPACE;
@@ -94,7 +95,7 @@ extern "C" int drk_pg_logprob_fwd_noalloc(const void* hidden, const void* W, int
     SimtFwdArgs a{hidden, W, in_dtype, ids, T, H, V, logp, lse, part, tgt, nsplit, status};
     rc = launch_simt_fwd(a, st);
   } else {
-    UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, part, tgt, nsplit, status};
+    UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, part, tgt, nsplit, status, ctas};
     rc = launch_umma_fwd(a, st);
   }
   if (rc != DRK_OK) g_launches = 0;

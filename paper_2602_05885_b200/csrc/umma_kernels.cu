@@ -28,14 +28,14 @@ namespace drk {
 
 namespace {
 
-constexpr int TM = 128, TN = 256, TK = 64, STAGES = 4;
-constexpr int A_BYTES = TM * TK * 2;  // 16 KiB
-constexpr int B_BYTES = TN * TK * 2;  // 32 KiB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int SUB_BYTES = 64 * TK * 2;  // one 64-wide MN-major box: 64 k-rows x 128 B
+constexpr int TM = 128, TN = 256, TK = 64;
+constexpr int A_BYTES = TM * TK * 2;      // 16 KiB: 128 rows of A per CTA
+constexpr int RING_BYTES = 192 * 1024;    // operand ring: 4 stages of 48 KiB, or 6 of 32 KiB for a CTA pair
+constexpr int MAX_STAGES = 6;
+constexpr int SUB_BYTES = 64 * TK * 2;    // one 64-wide MN-major box: 64 k-rows x 128 B
 constexpr int NUM_THREADS = 192;
-constexpr int NUM_BARS = 2 * STAGES + 5;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + NUM_BARS * 8 + 16;
+constexpr int NUM_BARS = 2 * MAX_STAGES + 5;
+constexpr int SMEM_BYTES = RING_BYTES + 1024 /*alignment slack*/ + NUM_BARS * 8 + 16;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;  // 2 s: far above any legitimate wait
 constexpr uint64_t DRAIN_LIMIT_NS = 20000000ull;   // 20 ms per outstanding copy when giving up
 constexpr float kLog2e = 1.4426950408889634f;
@@ -163,51 +163,67 @@ __device__ __forceinline__ void store_row_chunk(const UmmaParams& p, int64_t row
   }
 }
 
-template <int MODE>
+// CTAS = 1: one CTA per 128x256 tile.  CTAS = 2: a pair of CTAs (cluster of two) shares a 256x256
+// tile through tcgen05 cta_group::2: each CTA loads its 128 rows of A and its 128 of B's 256 rows,
+// the even CTA issues the MMAs for both, and each CTA drains its own 128 accumulator rows.
+template <int MODE, int CTAS>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const UmmaParams p) {
   constexpr bool A_MN = (MODE == DW);
   constexpr bool B_MN = (MODE == DW || MODE == DH);
-  constexpr uint32_t IDESC = ptx::make_idesc_bf16(TM, TN, A_MN ? 1 : 0, B_MN ? 1 : 0);
+  constexpr uint32_t IDESC = ptx::make_idesc_bf16(TM * CTAS, TN, A_MN ? 1 : 0, B_MN ? 1 : 0);
+  constexpr int BN_CTA = TN / CTAS;                 // rows of B this CTA loads
+  constexpr int B_BYTES_CTA = BN_CTA * TK * 2;
+  constexpr int STAGE = A_BYTES + B_BYTES_CTA;      // bytes per stage in this CTA
+  constexpr int NSTAGE = RING_BYTES / STAGE;        // 4 (one CTA) or 6 (pair)
+  constexpr uint32_t TX_BYTES = STAGE * CTAS;       // both CTAs' loads are credited to one barrier
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = ptx::smem_u32(smem_raw);
   const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
   uint8_t* smem = smem_raw + pad;
   const uint32_t smem_base = raw_addr + pad;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
-  const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + RING_BYTES);
+  const uint32_t bar_base = smem_base + RING_BYTES;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
-  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
-  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
-  const uint32_t done_bar = bar_base + 8u * (2 * STAGES + 4);
+  auto empty_bar = [&](int s) { return bar_base + 8u * (MAX_STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + 2 + a); };
+  const uint32_t done_bar = bar_base + 8u * (2 * MAX_STAGES + 4);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NUM_BARS);
   volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
   const int lane = threadIdx.x & 31;
+  const int cta_rank = (CTAS == 2) ? (int)ptx::cluster_ctarank() : 0;
+  const bool leader = (cta_rank == 0);
+  const int first_unit = blockIdx.x / CTAS, unit_stride = gridDim.x / CTAS;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) {
+    for (int s = 0; s < NSTAGE; ++s) {
       ptx::mbar_init(full_bar(s), 1);
       ptx::mbar_init(empty_bar(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(tfull_bar(a), 1);
-      ptx::mbar_init(tempty_bar(a), 4);
+      ptx::mbar_init(tempty_bar(a), 4 * CTAS);
     }
     ptx::mbar_init(done_bar, 1);
     *abort = 0;
     ptx::fence_barrier_init();
   }
   if (warp == 1) {
-    ptx::tmem_alloc(ptx::smem_u32(tmem_slot), 512);
-    ptx::tmem_relinquish();
+    if constexpr (CTAS == 2) {
+      ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), 512);
+      ptx::tmem_relinquish_pair();
+    } else {
+      ptx::tmem_alloc(ptx::smem_u32(tmem_slot), 512);
+      ptx::tmem_relinquish();
+    }
   }
   ptx::tc_fence_before();
-  __syncthreads();
+  if constexpr (CTAS == 2) ptx::cluster_sync(); else __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -218,48 +234,56 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       ptx::prefetch_tensormap(&tmB);
       uint32_t it = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < p.num_units && ok; u += gridDim.x) {
+      auto load = [&](uint32_t dst, const void* map, uint32_t bar, int x, int y) {
+        if constexpr (CTAS == 2) ptx::tma_load_2d_pair(dst, map, bar, x, y);
+        else ptx::tma_load_2d(dst, map, bar, x, y);
+      };
+      for (int u = first_unit; u < p.num_units && ok; u += unit_stride) {
         const Unit un = decode_unit(p, u);
+        const int a_row = (un.m * CTAS + cta_rank) * TM;   // first A row (M index) of this CTA
         for (int n = un.n_begin; n < un.n_end && ok; ++n) {
+          const int b_row = n * TN + cta_rank * BN_CTA;     // first B row (N index) of this CTA
           for (int kb = 0; kb < p.k_blocks; ++kb) {
-            const int s = it % STAGES;
-            const uint32_t ph = (it / STAGES) & 1u;
+            const int s = it % NSTAGE;
+            const uint32_t ph = (it / NSTAGE) & 1u;
             if (!ptx::mbar_wait(empty_bar(s), ph ^ 1u, abort, WAIT_LIMIT_NS)) { ok = false; break; }
-            ptx::mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES);
-            const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
+            if (leader) ptx::mbar_arrive_expect_tx(full_bar(s), TX_BYTES);
+            const uint32_t sa = smem_base + s * STAGE, sb = sa + A_BYTES;
             if constexpr (MODE == FWD || MODE == DL) {
-              ptx::tma_load_2d(sa, &tmA, full_bar(s), kb * TK, un.m * TM);
-              ptx::tma_load_2d(sb, &tmB, full_bar(s), kb * TK, p.v0 + n * TN);
+              load(sa, &tmA, full_bar(s), kb * TK, a_row);
+              load(sb, &tmB, full_bar(s), kb * TK, p.v0 + b_row);
             } else if constexpr (MODE == DW) {
 #pragma unroll
-              for (int j = 0; j < TM / 64; ++j)
-                ptx::tma_load_2d(sa + j * SUB_BYTES, &tmA, full_bar(s), un.m * TM + 64 * j, kb * TK);
+              for (int j = 0; j < TM / 64; ++j) load(sa + j * SUB_BYTES, &tmA, full_bar(s), a_row + 64 * j, kb * TK);
 #pragma unroll
-              for (int j = 0; j < TN / 64; ++j)
-                ptx::tma_load_2d(sb + j * SUB_BYTES, &tmB, full_bar(s), n * TN + 64 * j, kb * TK);
+              for (int j = 0; j < BN_CTA / 64; ++j) load(sb + j * SUB_BYTES, &tmB, full_bar(s), b_row + 64 * j, kb * TK);
             } else {  // DH
-              ptx::tma_load_2d(sa, &tmA, full_bar(s), kb * TK, un.m * TM);
+              load(sa, &tmA, full_bar(s), kb * TK, a_row);
 #pragma unroll
-              for (int j = 0; j < TN / 64; ++j)
-                ptx::tma_load_2d(sb + j * SUB_BYTES, &tmB, full_bar(s), n * TN + 64 * j, p.v0 + kb * TK);
+              for (int j = 0; j < BN_CTA / 64; ++j)
+                load(sb + j * SUB_BYTES, &tmB, full_bar(s), b_row + 64 * j, p.v0 + kb * TK);
             }
             ++it;
           }
         }
       }
-      if (!ok) {
-        // wait (bounded) for the copies still in flight before the block leaves
-        const uint32_t first = it > STAGES ? it - STAGES : 0;
+      if (!ok && leader) {
+        // wait (bounded) for the copies still in flight before the block leaves (a pair's loads are
+        // all credited to the even CTA's barriers; the odd CTA waits for its peer at the cluster barrier)
+        const uint32_t first = it > (uint32_t)NSTAGE ? it - NSTAGE : 0;
         for (uint32_t j = first; j < it; ++j)
-          ptx::mbar_wait(full_bar(j % STAGES), (j / STAGES) & 1u, nullptr, DRAIN_LIMIT_NS);
+          ptx::mbar_wait(full_bar(j % NSTAGE), (j / NSTAGE) & 1u, nullptr, DRAIN_LIMIT_NS);
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer (even CTA of a pair)
+    if (lane == 0 && leader) {
       uint32_t it = 0, tc = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < p.num_units && ok; u += gridDim.x) {
+      auto commit = [&](uint32_t bar) {
+        if constexpr (CTAS == 2) ptx::mma_commit_pair(bar, (uint16_t)3); else ptx::mma_commit(bar);
+      };
+      for (int u = first_unit; u < p.num_units && ok; u += unit_stride) {
         const Unit un = decode_unit(p, u);
         for (int n = un.n_begin; n < un.n_end && ok; ++n) {
           const int acc = tc & 1;
@@ -268,11 +292,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           ptx::tc_fence_after();
           const uint32_t d_tmem = tmem_base + acc * TN;
           for (int kb = 0; kb < p.k_blocks; ++kb) {
-            const int s = it % STAGES;
-            const uint32_t ph = (it / STAGES) & 1u;
+            const int s = it % NSTAGE;
+            const uint32_t ph = (it / NSTAGE) & 1u;
             if (!ptx::mbar_wait(full_bar(s), ph, abort, WAIT_LIMIT_NS)) { ok = false; break; }
             ptx::tc_fence_after();
-            const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
+            const uint32_t sa = smem_base + s * STAGE, sb = sa + A_BYTES;
 #pragma unroll
             for (int k = 0; k < TK / 16; ++k) {
               // K-major: 16 elements = 32 B further along the swizzled 128 B row.
@@ -281,18 +305,19 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                        : ptx::make_smem_desc(sa + k * 32, 16, 1024);
               const uint64_t db = B_MN ? ptx::make_smem_desc(sb + k * 2048, SUB_BYTES, 1024)
                                        : ptx::make_smem_desc(sb + k * 32, 16, 1024);
-              ptx::mma_bf16_ss(d_tmem, da, db, IDESC, (kb | k) != 0 ? 1u : 0u);
+              if constexpr (CTAS == 2) ptx::mma_bf16_ss_pair(d_tmem, da, db, IDESC, (kb | k) != 0 ? 1u : 0u);
+              else ptx::mma_bf16_ss(d_tmem, da, db, IDESC, (kb | k) != 0 ? 1u : 0u);
             }
-            ptx::mma_commit(empty_bar(s));  // frees the stage once these MMAs have read it
+            commit(empty_bar(s));  // frees the stage (in both CTAs) once these MMAs have read it
             ++it;
           }
           if (!ok) break;
-          ptx::mma_commit(tfull_bar(acc));  // accumulator complete
+          commit(tfull_bar(acc));  // accumulator complete (in both CTAs)
           ++tc;
         }
       }
       if (!ok) {
-        ptx::mma_commit(done_bar);
+        if constexpr (CTAS == 2) ptx::mma_commit_pair(done_bar, (uint16_t)1); else ptx::mma_commit(done_bar);
         ptx::mbar_wait(done_bar, 0, nullptr, DRAIN_LIMIT_NS);
       }
     }
@@ -301,9 +326,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int q = warp & 3;  // tensor-memory lane quarter this warp may read
     uint32_t tc = 0;
     bool ok = true;
-    for (int u = blockIdx.x; u < p.num_units && ok; u += gridDim.x) {
+    for (int u = first_unit; u < p.num_units && ok; u += unit_stride) {
       const Unit un = decode_unit(p, u);
-      const int64_t row = (int64_t)un.m * TM + q * 32 + lane;
+      const int64_t row = ((int64_t)un.m * CTAS + cta_rank) * TM + q * 32 + lane;
       const bool row_ok = row < p.rows;
       // per-unit state
       float run_m = -CUDART_INF_F, run_l = 0.f;  // FWD: log2-domain running max, sum
@@ -386,10 +411,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if (row_ok && col < p.cols) store_row_chunk(p, row, col, x);
           }
         }
-        // this warp has drained its quarter of the accumulator
+        // this warp has drained its quarter of the accumulator: tell the MMA issuer (even CTA)
         ptx::tc_fence_before();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+        if (lane == 0) {
+          if (CTAS == 2 && !leader) ptx::mbar_arrive_remote(tempty_bar(acc), 0);
+          else ptx::mbar_arrive(tempty_bar(acc));
+        }
         ++tc;
       }
       if (!ok) break;
@@ -405,11 +433,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   // ------------------------------------------------------------------ teardown
   ptx::tc_fence_before();
-  __syncthreads();
+  // In a pair neither CTA may leave (or free tensor memory) while its peer can still address it.
+  if constexpr (CTAS == 2) ptx::cluster_sync(); else __syncthreads();
   if (threadIdx.x == 0 && *abort) atomicOr(p.status, DRK_STATUS_TIMEOUT);
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, 512);
+    if constexpr (CTAS == 2) ptx::tmem_dealloc_pair(tmem_base, 512); else ptx::tmem_dealloc(tmem_base, 512);
   }
 }
 
@@ -456,24 +485,79 @@ int sm_count() {
   return n;
 }
 
-template <int MODE>
-int launch_mode(const CUtensorMap& a, const CUtensorMap& b, UmmaParams p, cudaStream_t st) {
+template <int MODE, int CTAS>
+__global__ void umma_gemm_kernel(const __grid_constant__ CUtensorMap, const __grid_constant__ CUtensorMap,
+                                 const UmmaParams);
+
+// How many two-CTA clusters of this kernel the device can hold at once (one CTA per SM).
+int resident_pairs() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return sm_count() / 2;
+  if (cached[dev] > 0) return cached[dev];
+  auto kern = umma_gemm_kernel<0, 2>;
+  int n = 0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(sm_count() / 2 * 2);
+  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
+      cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) {
+    (void)cudaGetLastError();
+    n = sm_count() / 2;
+  }
+  if (n > sm_count() / 2) n = sm_count() / 2;
+  cached[dev] = n;
+  return n;
+}
+
+template <int MODE, int CTAS>
+int launch_mode_ctas(const CUtensorMap& a, const CUtensorMap& b, UmmaParams p, cudaStream_t st) {
   p.num_units = p.m_tiles * p.nj;
   if (p.num_units <= 0) return DRK_OK;
-  DRK_CUDA_CHECK(cudaFuncSetAttribute(umma_gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
-  const int grid = p.num_units < sm_count() ? p.num_units : sm_count();
-  umma_gemm_kernel<MODE><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(a, b, p);
+  auto kern = umma_gemm_kernel<MODE, CTAS>;
+  DRK_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  if (CTAS == 2) {
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const int pairs = resident_pairs();
+    cfg.gridDim = dim3(2 * (p.num_units < pairs ? p.num_units : pairs));
+  } else {
+    cfg.gridDim = dim3(p.num_units < sm_count() ? p.num_units : sm_count());
+  }
+  if (cudaLaunchKernelEx(&cfg, kern, a, b, p) != cudaSuccess) { (void)cudaGetLastError(); return DRK_ERR_CUDA; }
   DRK_LAUNCHED();
   return DRK_OK;
 }
 
+template <int MODE>
+int launch_mode(int ctas, const CUtensorMap& a, const CUtensorMap& b, const UmmaParams& p, cudaStream_t st) {
+  return ctas == 2 ? launch_mode_ctas<MODE, 2>(a, b, p, st) : launch_mode_ctas<MODE, 1>(a, b, p, st);
+}
+
 }  // namespace
 
-int umma_nsplit(int64_t T, int V) {
-  const int64_t m_tiles = ceil_div(T, TM);
+int umma_nsplit(int64_t T, int V, int ctas) {
+  const int64_t m_tiles = ceil_div(T, TM * ctas);
   const int n_tiles = (int)ceil_div(V, TN);
   if (m_tiles <= 0) return 1;
-  const int sms = 148;
+  const int sms = 148 / ctas;
   int best = 1;
   double best_eff = -1.0;
   for (int ns = 1; ns <= 32 && ns <= n_tiles; ++ns) {
@@ -491,27 +575,31 @@ int umma_nsplit(int64_t T, int V) {
 }
 
 int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st) {
+  const int ctas = a.ctas == 2 ? 2 : 1;
   CUtensorMap mh, mw;
   if (!make_map(&mh, a.hidden, a.H, a.T, a.H, TK, TM)) return DRK_ERR_CUDA;
-  if (!make_map(&mw, a.W, a.H, a.V, a.H, TK, TN)) return DRK_ERR_CUDA;
+  if (!make_map(&mw, a.W, a.H, a.V, a.H, TK, TN / ctas)) return DRK_ERR_CUDA;
   UmmaParams p{};
-  p.m_tiles = (int)ceil_div(a.T, TM);
+  p.m_tiles = (int)ceil_div(a.T, TM * ctas);
   p.n_tiles = (int)ceil_div(a.V, TN);
   p.k_blocks = (int)ceil_div(a.H, TK);
   p.nj = a.nsplit;
   p.tiles_per_unit = (int)ceil_div(p.n_tiles, a.nsplit);
-  p.group_m = 148 / a.nsplit > 0 ? 148 / a.nsplit : 1;
+  const int slots = 148 / ctas;
+  p.group_m = slots / a.nsplit > 0 ? slots / a.nsplit : 1;
   p.rows = a.T; p.cols = a.V; p.v0 = 0; p.T = a.T;
   p.ids = a.ids; p.part = a.part; p.tgt = a.tgt; p.status = a.status;
-  int rc = launch_mode<FWD>(mh, mw, p, st);
+  int rc = launch_mode<FWD>(ctas, mh, mw, p, st);
   if (rc != DRK_OK) return rc;
   return launch_lse_merge(a.part, a.tgt, a.ids, a.T, a.V, a.nsplit, a.logp, a.lse, a.status, st);
 }
 
 int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {
+  const int ctas = a.ctas == 2 ? 2 : 1;
+  const int TMC = TM * ctas;   // rows of one work unit's tile
   CUtensorMap mh_k, mw_k, mh_mn, mw_mn;
   if (!make_map(&mh_k, a.hidden, a.H, a.T, a.H, TK, TM)) return DRK_ERR_CUDA;
-  if (!make_map(&mw_k, a.W, a.H, a.V, a.H, TK, TN)) return DRK_ERR_CUDA;
+  if (!make_map(&mw_k, a.W, a.H, a.V, a.H, TK, TN / ctas)) return DRK_ERR_CUDA;
   if (!make_map(&mh_mn, a.hidden, a.H, a.T, a.H, 64, TK)) return DRK_ERR_CUDA;
   if (!make_map(&mw_mn, a.W, a.H, a.V, a.H, 64, TK)) return DRK_ERR_CUDA;
   float* dh_acc = (a.dh_dtype == DRK_F32) ? (float*)a.dH : a.dH_acc;
@@ -524,42 +612,42 @@ int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {
     if (!make_map(&mdl_mn, a.dL, vc_this, a.T, a.vc, 64, TK)) return DRK_ERR_CUDA;
     {  // dL chunk = c (softmax - onehot), recomputed from hidden W^T
       UmmaParams p{};
-      p.m_tiles = (int)ceil_div(a.T, TM);
+      p.m_tiles = (int)ceil_div(a.T, TMC);
       p.n_tiles = (int)ceil_div(vc_this, TN);
       p.k_blocks = (int)ceil_div(a.H, TK);
-      p.nj = p.n_tiles; p.tiles_per_unit = 1; p.group_m = 16;
+      p.nj = p.n_tiles; p.tiles_per_unit = 1; p.group_m = 16 / ctas;
       p.rows = a.T; p.cols = vc_this; p.v0 = v0; p.T = a.T;
       p.ids = a.ids; p.lse = a.lse; p.coeff = a.coeff; p.dL = a.dL; p.vc = a.vc; p.status = a.status;
-      int rc = launch_mode<DL>(mh_k, mw_k, p, st);
+      int rc = launch_mode<DL>(ctas, mh_k, mw_k, p, st);
       if (rc != DRK_OK) return rc;
     }
     {  // dW[v0 : v0 + vc_this, :] (+)= dL^T hidden
       UmmaParams p{};
-      p.m_tiles = (int)ceil_div(vc_this, TM);
+      p.m_tiles = (int)ceil_div(vc_this, TMC);
       p.n_tiles = (int)ceil_div(a.H, TN);
       p.k_blocks = (int)ceil_div(a.T, TK);
-      p.nj = p.n_tiles; p.tiles_per_unit = 1; p.group_m = 16;
+      p.nj = p.n_tiles; p.tiles_per_unit = 1; p.group_m = 16 / ctas;
       p.rows = vc_this; p.cols = a.H; p.v0 = v0; p.T = a.T;
       const size_t esz = a.dw_dtype == DRK_BF16 ? 2 : 4;
       p.C = (char*)a.dW + (size_t)v0 * a.H * esz; p.C_in = p.C; p.ldc = a.H;
       p.beta = a.dw_accumulate; p.out_bf16 = a.dw_dtype == DRK_BF16; p.in_bf16 = p.out_bf16;
       p.status = a.status;
-      int rc = launch_mode<DW>(mdl_mn, mh_mn, p, st);
+      int rc = launch_mode<DW>(ctas, mdl_mn, mh_mn, p, st);
       if (rc != DRK_OK) return rc;
     }
     {  // dH (+)= dL W[v0 : v0 + vc_this, :]
       UmmaParams p{};
-      p.m_tiles = (int)ceil_div(a.T, TM);
+      p.m_tiles = (int)ceil_div(a.T, TMC);
       p.n_tiles = (int)ceil_div(a.H, TN);
       p.k_blocks = (int)ceil_div(vc_this, TK);
-      p.nj = p.n_tiles; p.tiles_per_unit = 1; p.group_m = 8;
+      p.nj = p.n_tiles; p.tiles_per_unit = 1; p.group_m = 8 / ctas;
       p.rows = a.T; p.cols = a.H; p.v0 = v0; p.T = a.T;
       const bool last = (chunk == n_chunks - 1);
       p.C_in = dh_acc; p.in_bf16 = 0; p.ldc = a.H; p.beta = chunk > 0;
       if (last && a.dh_dtype == DRK_BF16) { p.C = a.dH; p.out_bf16 = 1; }
       else { p.C = dh_acc; p.out_bf16 = 0; }
       p.status = a.status;
-      int rc = launch_mode<DH>(mdl_k, mw_mn, p, st);
+      int rc = launch_mode<DH>(ctas, mdl_k, mw_mn, p, st);
       if (rc != DRK_OK) return rc;
     }
   }

@@ -15,10 +15,11 @@ OPEN = (0.0, math.inf, 0.0)      # MRS switched off: every sample with a masked 
 
 
 @pytest.mark.parametrize("T,H,V", [(1, 64, 300), (127, 264, 4104), (129, 72, 4099), (300, 512, 257), (64, 8, 1)])
-@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
-def test_ragged_sizes(T, H, V, dtype):
+@pytest.mark.parametrize("dtype,engine", [(torch.bfloat16, B.DRK_ENGINE_AUTO), (torch.bfloat16, B.DRK_ENGINE_UMMA_1CTA),
+                                          (torch.float32, B.DRK_ENGINE_AUTO)])
+def test_ragged_sizes(T, H, V, dtype, engine):
     case = Hh.build_plain_case(f"r{T}_{H}_{V}", T=T, H=H, V=V, dtype=dtype, S=3, seed=T + V, mask_frac=0.2)
-    dev = run_device(case, make_params(*OPEN, v_chunk=256))
+    dev = run_device(case, make_params(*OPEN, v_chunk=256, engine=engine))
     assert dev["status"] == 0
     Hh.check_against_oracle(case, dev, *OPEN)
 

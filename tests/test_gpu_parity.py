@@ -73,7 +73,7 @@ def test_tiny_forward_only_and_determinism():
 
 
 @pytest.mark.parametrize("name", ["medium", "q8b", "q14b", "ragged"])
-@pytest.mark.parametrize("engine", [B.DRK_ENGINE_AUTO, B.DRK_ENGINE_SIMT])
+@pytest.mark.parametrize("engine", [B.DRK_ENGINE_AUTO, B.DRK_ENGINE_UMMA_1CTA, B.DRK_ENGINE_SIMT])
 def test_bf16_shapes(name, engine):
     if engine == B.DRK_ENGINE_SIMT and name in ("q14b", "ragged"):
         pytest.skip("FFMA cross-check runs on two bf16 shapes only (time)")
