@@ -165,6 +165,8 @@ def main():
     ap.add_argument("--dw-dtype", default="f32", choices=["f32", "bf16"])
     ap.add_argument("--dh-dtype", default="bf16", choices=["f32", "bf16"])
     ap.add_argument("--v-chunk", type=int, default=0)
+    ap.add_argument("--engine", default="auto", choices=["auto", "1cta"],
+                    help="auto: tcgen05 kernels on CTA pairs; 1cta: one CTA per tile")
     ap.add_argument("--mrs", default="wide", choices=["wide", "paper", "off"])
     ap.add_argument("--ref-tokens", type=int, default=256)
     ap.add_argument("--cpu-tokens", type=int, default=512)
@@ -204,6 +206,7 @@ def main():
     p.dw_dtype = B.DRK_BF16 if args.dw_dtype == "bf16" else B.DRK_F32
     p.dh_dtype = B.DRK_BF16 if args.dh_dtype == "bf16" else B.DRK_F32
     p.v_chunk = args.v_chunk
+    p.engine = B.DRK_ENGINE_UMMA_1CTA if args.engine == "1cta" else B.DRK_ENGINE_AUTO
     bufs = B.PgLossBuffers(T, H, V, S, code, p, dev)
     R, Tmax = wl.reward.shape
     ret = torch.empty_like(wl.reward)
@@ -263,7 +266,7 @@ def main():
         e1.record(stream)
         torch.cuda.synchronize()
         call_ms.append(e0.elapsed_time(e1))
-    n_gemm_launches = B.drk_last_launch_count() - 5     # all but merge + 3 MRS kernels + (bf16 dH: none extra)
+    n_gemm_launches = B.drk_last_launch_count() - 4     # all but the merge and the three MRS kernels
     fused_ms = statistics.mean(call_ms)
     flops = 8.0 * T * H * V
     peaks = measured_peaks()
@@ -319,6 +322,7 @@ def main():
             "config": {"workload": f"{wl.name}-shaped packed micro-batch", "T": T, "H": H, "V": V, "segments": S,
                        "rollout_batch": f"{R} rollouts x {Tmax} turns", "mrs": args.mrs,
                        "dW": args.dw_dtype, "dH": args.dh_dtype, "v_chunk": args.v_chunk or "default",
+                       "engine": args.engine,
                        "l2": "inputs exceed L2 (W alone is %.2f GB); no flush" % (V * H * 2 / 1e9),
                        "parallelism": f"dp{world}: one micro-batch per rank, no collective on the loss path"},
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s",
