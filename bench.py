@@ -257,20 +257,44 @@ def main():
     # ---------------------------------------------------------------- the fused call alone (roofline)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     seg_adv = adv.view(-1).index_select(0, seg_flat)
-    call_ms = []
-    for _ in range(min(args.steps, 5)):
-        e0.record(stream)
-        B.drk_pg_loss_fwd_bwd(wl.hidden, wl.W, code, wl.ids, wl.rollout_logp, wl.loss_mask, wl.cu, seg_adv, T, H, V, S,
-                              p, bufs.loss, bufs.logp, bufs.lse, bufs.seg_w, bufs.seg_keep, bufs.counters, bufs.dH,
-                              bufs.dW, bufs.workspace, bufs.workspace_bytes, bufs.status, stream)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        call_ms.append(e0.elapsed_time(e1))
-    n_gemm_launches = B.drk_last_launch_count() - 4     # all but the merge and the three MRS kernels
-    fused_ms = statistics.mean(call_ms)
-    flops = 8.0 * T * H * V
+
+    def time_fused(pp, reps):
+        out = []
+        for _ in range(reps):
+            e0.record(stream)
+            B.drk_pg_loss_fwd_bwd(wl.hidden, wl.W, code, wl.ids, wl.rollout_logp, wl.loss_mask, wl.cu, seg_adv, T, H,
+                                  V, S, pp, bufs.loss, bufs.logp, bufs.lse, bufs.seg_w, bufs.seg_keep, bufs.counters,
+                                  bufs.dH, bufs.dW, bufs.workspace, bufs.workspace_bytes, bufs.status, stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            out.append(e0.elapsed_time(e1))
+        return statistics.mean(out)
+
+    def backward_rows():
+        # rows the backward GEMMs process: loss-masked tokens of retained samples with a non-zero advantage
+        keep = bufs.seg_keep.bool() & (seg_adv != 0)
+        cu = wl.cu.long()
+        csum = torch.cat([torch.zeros(1, dtype=torch.long, device=dev), wl.loss_mask.long().cumsum(0)])
+        per_seg = csum[cu[1:]] - csum[cu[:-1]]
+        return int((per_seg * keep.long()).sum().item())
+
+    fused_ms = time_fused(p, min(args.steps, 5))
+    # merge + 3 MRS + 4 compaction kernels are not GEMM launches (the FFMA path has no compaction)
+    n_gemm_launches = B.drk_last_launch_count() - (8 if code == B.DRK_BF16 else 4)
+    Tc = backward_rows() if code == B.DRK_BF16 else T
+    flops = (2.0 * T + 6.0 * Tc) * H * V
     peaks = measured_peaks()
     achieved = flops / (fused_ms * 1e-3) / 1e12
+    # the same call with rejection switched off: every loss-masked token goes through the backward
+    p_off = B.drk_pg_params_default()
+    ctypes_copy = [f[0] for f in p._fields_]
+    for f in ctypes_copy:
+        setattr(p_off, f, getattr(p, f))
+    p_off.mrs_lo, p_off.mrs_hi, p_off.veto_ratio = 0.0, float("inf"), 0.0
+    off_ms = time_fused(p_off, min(args.steps, 5))
+    Tc_off = backward_rows() if code == B.DRK_BF16 else T
+    off_tflops = (2.0 * T + 6.0 * Tc_off) * H * V / (off_ms * 1e-3) / 1e12
+    time_fused(p, 1)   # leave the outputs of the configured run in the buffers
 
     # ---------------------------------------------------------------- end to end with host buffers
     e2e = None
@@ -329,6 +353,12 @@ def main():
                          "frac": achieved / peaks["tflops"], "traffic": None,
                          "kernel": "umma_gemm_kernel (all four instantiations inside one drk_pg_loss_fwd_bwd call)",
                          "flops_per_call": flops, "call_ms": fused_ms, "gemm_launches_per_call": n_gemm_launches,
+                         "flops_rule": "(2 T + 6 Tc) H V: forward over all T rows, backward over the Tc rows with "
+                                       "a non-zero coefficient (rows of rejected or masked tokens are skipped)",
+                         "rows_in_backward": Tc,
+                         "no_rejection": {"call_ms": off_ms, "rows_in_backward": Tc_off, "tflops": off_tflops,
+                                          "frac": off_tflops / peaks["tflops"],
+                                          "tokens_per_s": T / (off_ms * 1e-3)},
                          "peak_source": f"bf16_tflops_sustained of {peaks['source']}",
                          "frac_of_burst": achieved / peaks["burst"], "frac_of_nominal_2250": achieved / 2250.0},
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": n_launch, "clocks": clocks,

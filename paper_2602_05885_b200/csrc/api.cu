@@ -33,11 +33,11 @@ bool sizes_ok(int64_t T, int H, int V, int in_dtype) {
 // Chunk width for the tensor-core backward when the caller leaves it to the library: the multiple of
 // 256 that minimises the modelled time of the three per-chunk kernels.  Each kernel is persistent
 // over 148 SMs with 128x256 tiles, so its time is (waves of tiles) x (k-blocks per tile); a fixed
-// cost per launch stands for fill and drain.  The dL buffer is kept below ~1 GiB.
+// cost per launch stands for fill and drain.  The dL buffer is kept below ~512 MiB (or 8192 columns).
 int auto_vchunk(int64_t T, int H, int V) {
   const int64_t sms = 148, launch_cost = 96;
   const int64_t mt_T = ceil_div(T, 128), nt_H = ceil_div(H, 256), kb_H = ceil_div(H, 64), kb_T = ceil_div(T, 64);
-  int64_t cap = ((int64_t)1 << 30) / (2 * (T > 0 ? T : 1)) / 256 * 256;
+  int64_t cap = ((int64_t)1 << 29) / (2 * (T > 0 ? T : 1)) / 256 * 256;
   if (cap < 8192) cap = 8192;
   if (cap > 32768) cap = 32768;
   const int64_t vmax = ceil_div(V, 256) * 256;
@@ -95,14 +95,31 @@ struct BwdWs {
   void* dL;
   float* dH_acc;
   int vc;
+  // tensor-core path only: compaction of the rows with non-zero coefficient
+  int32_t* blk_cnt;
+  int32_t* blk_off;
+  int32_t* n_rows;
+  int32_t* rowmap;
+  __nv_bfloat16* hidden_c;
 };
 BwdWs carve_bwd(Carver& c, int64_t T, int H, int V, int S, bool simt, const drk_pg_params& p) {
   BwdWs w;
   w.vc = round_vchunk(p.v_chunk, T, H, V, simt);
   w.coeff = static_cast<float*>(c.take(sizeof(float) * (size_t)T));
   w.seg_stats = static_cast<double*>(c.take(sizeof(double) * 4 * (size_t)S));
-  w.dL = c.take((simt ? 4 : 2) * (size_t)T * (size_t)w.vc);
+  const size_t rows_cap = (size_t)(ceil_div(T, 256) * 256);   // dL also holds the zero rows that pad the last tile
+  w.dL = c.take((simt ? 4 : 2) * (simt ? (size_t)T : rows_cap) * (size_t)w.vc);
   w.dH_acc = (p.dh_dtype == DRK_BF16) ? static_cast<float*>(c.take(sizeof(float) * (size_t)T * (size_t)H)) : nullptr;
+  w.blk_cnt = w.blk_off = w.n_rows = w.rowmap = nullptr;
+  w.hidden_c = nullptr;
+  if (!simt) {
+    const size_t nblk = (size_t)compact_blocks(T), len = (size_t)compact_map_len(T);
+    w.blk_cnt = static_cast<int32_t*>(c.take(sizeof(int32_t) * nblk));
+    w.blk_off = static_cast<int32_t*>(c.take(sizeof(int32_t) * nblk));
+    w.n_rows = static_cast<int32_t*>(c.take(sizeof(int32_t) * 2));
+    w.rowmap = static_cast<int32_t*>(c.take(sizeof(int32_t) * len));
+    w.hidden_c = static_cast<__nv_bfloat16*>(c.take(2 * len * (size_t)H));
+  }
   return w;
 }
 
@@ -260,8 +277,13 @@ int drk_pg_loss_fwd_bwd(const void* hidden, const void* W, int32_t in_dtype, con
                   dH, p.dh_dtype, bw.dH_acc, dW, p.dw_dtype, p.dw_accumulate};
     rc = launch_simt_bwd(b, st);
   } else {
+    CompactArgs ca{bw.coeff, static_cast<const __nv_bfloat16*>(hidden), T, H, bw.blk_cnt, bw.blk_off, bw.n_rows,
+                   bw.rowmap, bw.hidden_c};
+    rc = launch_compact(ca, st);
+    if (rc != DRK_OK) return fail(rc);
     UmmaBwdArgs b{hidden, W, ids, T, H, V, lse, bw.coeff, static_cast<__nv_bfloat16*>(bw.dL), bw.vc,
-                  dH, p.dh_dtype, bw.dH_acc, dW, p.dw_dtype, p.dw_accumulate, status, umma_ctas(p.engine)};
+                  dH, p.dh_dtype, bw.dH_acc, dW, p.dw_dtype, p.dw_accumulate, status, umma_ctas(p.engine),
+                  bw.hidden_c, bw.rowmap, bw.n_rows};
     rc = launch_umma_bwd(b, st);
   }
   if (rc != DRK_OK) return fail(rc);

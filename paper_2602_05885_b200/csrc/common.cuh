@@ -76,8 +76,19 @@ struct UmmaBwdArgs {
   const float* lse; const float* coeff; __nv_bfloat16* dL /*[T*vc]*/; int vc;
   void* dH; int dh_dtype; float* dH_acc; void* dW; int dw_dtype; int dw_accumulate; uint32_t* status;
   int ctas;
+  const __nv_bfloat16* hidden_c; const int32_t* rowmap; const int32_t* n_rows;  // compacted rows
 };
 int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st);
+
+// Compaction of the rows with non-zero coefficient (backward pass of the tensor-core path).
+struct CompactArgs {
+  const float* coeff; const __nv_bfloat16* hidden; int64_t T; int H;
+  int32_t* blk_cnt; int32_t* blk_off; int32_t* n_rows /*[2]: count, count rounded up to 256*/;
+  int32_t* rowmap /*[compact_map_len(T)]*/; __nv_bfloat16* hidden_c /*[compact_map_len(T), H]*/;
+};
+int64_t compact_map_len(int64_t T);
+int compact_blocks(int64_t T);
+int launch_compact(const CompactArgs& a, cudaStream_t st);
 
 // Small utility kernels.
 int launch_f32_to_bf16(const float* src, __nv_bfloat16* dst, size_t n, cudaStream_t st);

@@ -61,17 +61,21 @@ struct UmmaParams {
   int64_t ldc;
   int beta, out_bf16, in_bf16;
   uint32_t* status;
+  // Compacted backward: the row dimension (M for DL and DH, K for DW) runs over the rows listed in
+  // rowmap; their number is n_rows[0] (n_rows[1] = rounded up to 256), known on the device only.
+  const int32_t* rowmap;
+  const int32_t* n_rows;
 };
 
 struct Unit {
   int m, j, n_begin, n_end;
 };
 
-__device__ __forceinline__ Unit decode_unit(const UmmaParams& p, int u) {
+__device__ __forceinline__ Unit decode_unit(const UmmaParams& p, int m_tiles, int u) {
   const int per_group = p.group_m * p.nj;
   const int g = u / per_group;
   const int rem = u - g * per_group;
-  const int gm = min(p.group_m, p.m_tiles - g * p.group_m);
+  const int gm = min(p.group_m, m_tiles - g * p.group_m);
   Unit r;
   r.j = rem / gm;
   r.m = g * p.group_m + rem % gm;
@@ -200,6 +204,19 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const bool leader = (cta_rank == 0);
   const int first_unit = blockIdx.x / CTAS, unit_stride = gridDim.x / CTAS;
 
+  // Work extents: fixed by the host, or derived from the device-side count of compacted rows.
+  int m_tiles = p.m_tiles, k_blocks = p.k_blocks;
+  int64_t rows = p.rows;
+  if (p.n_rows != nullptr) {
+    const int cnt = p.n_rows[0];
+    if constexpr (MODE == DL || MODE == DH) {
+      m_tiles = (cnt + TM * CTAS - 1) / (TM * CTAS);
+      rows = p.n_rows[1];
+    }
+    if constexpr (MODE == DW) k_blocks = (cnt + TK - 1) / TK;
+  }
+  const int num_units = m_tiles * p.nj;
+
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSTAGE; ++s) {
       ptx::mbar_init(full_bar(s), 1);
@@ -238,12 +255,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if constexpr (CTAS == 2) ptx::tma_load_2d_pair(dst, map, bar, x, y);
         else ptx::tma_load_2d(dst, map, bar, x, y);
       };
-      for (int u = first_unit; u < p.num_units && ok; u += unit_stride) {
-        const Unit un = decode_unit(p, u);
+      for (int u = first_unit; u < num_units && ok; u += unit_stride) {
+        const Unit un = decode_unit(p, m_tiles, u);
         const int a_row = (un.m * CTAS + cta_rank) * TM;   // first A row (M index) of this CTA
         for (int n = un.n_begin; n < un.n_end && ok; ++n) {
           const int b_row = n * TN + cta_rank * BN_CTA;     // first B row (N index) of this CTA
-          for (int kb = 0; kb < p.k_blocks; ++kb) {
+          for (int kb = 0; kb < k_blocks; ++kb) {
             const int s = it % NSTAGE;
             const uint32_t ph = (it / NSTAGE) & 1u;
             if (!ptx::mbar_wait(empty_bar(s), ph ^ 1u, abort, WAIT_LIMIT_NS)) { ok = false; break; }
@@ -283,15 +300,15 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       auto commit = [&](uint32_t bar) {
         if constexpr (CTAS == 2) ptx::mma_commit_pair(bar, (uint16_t)3); else ptx::mma_commit(bar);
       };
-      for (int u = first_unit; u < p.num_units && ok; u += unit_stride) {
-        const Unit un = decode_unit(p, u);
+      for (int u = first_unit; u < num_units && ok; u += unit_stride) {
+        const Unit un = decode_unit(p, m_tiles, u);
         for (int n = un.n_begin; n < un.n_end && ok; ++n) {
           const int acc = tc & 1;
           const uint32_t aph = (tc >> 1) & 1u;
           if (!ptx::mbar_wait(tempty_bar(acc), aph ^ 1u, abort, WAIT_LIMIT_NS)) { ok = false; break; }
           ptx::tc_fence_after();
           const uint32_t d_tmem = tmem_base + acc * TN;
-          for (int kb = 0; kb < p.k_blocks; ++kb) {
+          for (int kb = 0; kb < k_blocks; ++kb) {
             const int s = it % NSTAGE;
             const uint32_t ph = (it / NSTAGE) & 1u;
             if (!ptx::mbar_wait(full_bar(s), ph, abort, WAIT_LIMIT_NS)) { ok = false; break; }
@@ -326,19 +343,25 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int q = warp & 3;  // tensor-memory lane quarter this warp may read
     uint32_t tc = 0;
     bool ok = true;
-    for (int u = first_unit; u < p.num_units && ok; u += unit_stride) {
-      const Unit un = decode_unit(p, u);
+    for (int u = first_unit; u < num_units && ok; u += unit_stride) {
+      const Unit un = decode_unit(p, m_tiles, u);
       const int64_t row = ((int64_t)un.m * CTAS + cta_rank) * TM + q * 32 + lane;
-      const bool row_ok = row < p.rows;
+      bool row_ok = row < rows;
+      // orow: the token this accumulator row belongs to (differs from row when rows are compacted)
+      int64_t orow = row;
+      if constexpr (MODE == DL || MODE == DH) {
+        if (p.rowmap != nullptr) orow = row_ok ? (int64_t)p.rowmap[row] : -1;
+        if constexpr (MODE == DH) row_ok = row_ok && orow >= 0;
+      }
       // per-unit state
       float run_m = -CUDART_INF_F, run_l = 0.f;  // FWD: log2-domain running max, sum
       int id = -1;
       float c_t = 0.f, z2 = 0.f;
-      if constexpr (MODE == FWD || MODE == DL) {
+      if constexpr (MODE == FWD) {
         if (row_ok) id = p.ids[row];
       }
       if constexpr (MODE == DL) {
-        if (row_ok) { c_t = p.coeff[row]; z2 = p.lse[row] * kLog2e; }
+        if (row_ok && orow >= 0) { id = p.ids[orow]; c_t = p.coeff[orow]; z2 = p.lse[orow] * kLog2e; }
       }
       for (int n = un.n_begin; n < un.n_end; ++n) {
         const int acc = tc & 1;
@@ -408,7 +431,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               }
             }
           } else {  // DW, DH
-            if (row_ok && col < p.cols) store_row_chunk(p, row, col, x);
+            if constexpr (MODE == DW) {
+              if (k_blocks == 0) {  // nothing to contract over: the accumulator was never written
+#pragma unroll
+                for (int j = 0; j < 32; ++j) x[j] = 0.f;
+              }
+            }
+            if (row_ok && col < p.cols) store_row_chunk(p, orow, col, x);
           }
         }
         // this warp has drained its quarter of the accumulator: tell the MMA issuer (even CTA)
@@ -520,7 +549,7 @@ int resident_pairs() {
 
 template <int MODE, int CTAS>
 int launch_mode_ctas(const CUtensorMap& a, const CUtensorMap& b, UmmaParams p, cudaStream_t st) {
-  p.num_units = p.m_tiles * p.nj;
+  p.num_units = p.m_tiles * p.nj;   // upper bound when the row count lives on the device
   if (p.num_units <= 0) return DRK_OK;
   auto kern = umma_gemm_kernel<MODE, CTAS>;
   DRK_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
@@ -597,19 +626,24 @@ int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st) {
 int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {
   const int ctas = a.ctas == 2 ? 2 : 1;
   const int TMC = TM * ctas;   // rows of one work unit's tile
+  // The row dimension of the three contractions runs over the compacted rows (hidden_c, rowmap);
+  // buffers are sized for the worst case (every row kept), the kernels read the actual count.
+  const int64_t rows_cap = ceil_div(a.T, 256) * 256;
   CUtensorMap mh_k, mw_k, mh_mn, mw_mn;
-  if (!make_map(&mh_k, a.hidden, a.H, a.T, a.H, TK, TM)) return DRK_ERR_CUDA;
+  if (!make_map(&mh_k, a.hidden_c, a.H, rows_cap, a.H, TK, TM)) return DRK_ERR_CUDA;
   if (!make_map(&mw_k, a.W, a.H, a.V, a.H, TK, TN / ctas)) return DRK_ERR_CUDA;
-  if (!make_map(&mh_mn, a.hidden, a.H, a.T, a.H, 64, TK)) return DRK_ERR_CUDA;
+  if (!make_map(&mh_mn, a.hidden_c, a.H, rows_cap, a.H, 64, TK)) return DRK_ERR_CUDA;
   if (!make_map(&mw_mn, a.W, a.H, a.V, a.H, 64, TK)) return DRK_ERR_CUDA;
   float* dh_acc = (a.dh_dtype == DRK_F32) ? (float*)a.dH : a.dH_acc;
+  // rows that are not in the compacted set keep this zero
+  DRK_CUDA_CHECK(cudaMemsetAsync(a.dH, 0, (size_t)a.T * a.H * (a.dh_dtype == DRK_BF16 ? 2 : 4), st));
   const int n_chunks = (int)ceil_div(a.V, a.vc);
   int chunk = 0;
   for (int v0 = 0; v0 < a.V; v0 += a.vc, ++chunk) {
     const int vc_this = a.V - v0 < a.vc ? a.V - v0 : a.vc;
     CUtensorMap mdl_k, mdl_mn;
-    if (!make_map(&mdl_k, a.dL, vc_this, a.T, a.vc, TK, TM)) return DRK_ERR_CUDA;
-    if (!make_map(&mdl_mn, a.dL, vc_this, a.T, a.vc, 64, TK)) return DRK_ERR_CUDA;
+    if (!make_map(&mdl_k, a.dL, vc_this, rows_cap, a.vc, TK, TM)) return DRK_ERR_CUDA;
+    if (!make_map(&mdl_mn, a.dL, vc_this, rows_cap, a.vc, 64, TK)) return DRK_ERR_CUDA;
     {  // dL chunk = c (softmax - onehot), recomputed from hidden W^T
       UmmaParams p{};
       p.m_tiles = (int)ceil_div(a.T, TMC);
@@ -618,6 +652,7 @@ int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {
       p.nj = p.n_tiles; p.tiles_per_unit = 1; p.group_m = 16 / ctas;
       p.rows = a.T; p.cols = vc_this; p.v0 = v0; p.T = a.T;
       p.ids = a.ids; p.lse = a.lse; p.coeff = a.coeff; p.dL = a.dL; p.vc = a.vc; p.status = a.status;
+      p.rowmap = a.rowmap; p.n_rows = a.n_rows;
       int rc = launch_mode<DL>(ctas, mh_k, mw_k, p, st);
       if (rc != DRK_OK) return rc;
     }
@@ -632,6 +667,7 @@ int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {
       p.C = (char*)a.dW + (size_t)v0 * a.H * esz; p.C_in = p.C; p.ldc = a.H;
       p.beta = a.dw_accumulate; p.out_bf16 = a.dw_dtype == DRK_BF16; p.in_bf16 = p.out_bf16;
       p.status = a.status;
+      p.rowmap = a.rowmap; p.n_rows = a.n_rows;
       int rc = launch_mode<DW>(ctas, mdl_mn, mh_mn, p, st);
       if (rc != DRK_OK) return rc;
     }
@@ -647,6 +683,7 @@ int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {
       if (last && a.dh_dtype == DRK_BF16) { p.C = a.dH; p.out_bf16 = 1; }
       else { p.C = dh_acc; p.out_bf16 = 0; }
       p.status = a.status;
+      p.rowmap = a.rowmap; p.n_rows = a.n_rows;
       int rc = launch_mode<DH>(ctas, mdl_k, mw_mn, p, st);
       if (rc != DRK_OK) return rc;
     }
