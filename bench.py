@@ -154,6 +154,57 @@ def cpu_baseline(n_tok: int):
                       "(fp64: TRLOO + full logits + log-softmax + MRS + loss + dH + dW)"}
 
 
+def run_sweep(args):
+    """Roofline sweep: T x V x H grid, bf16, equal-length segments, uniform ids.  One JSON line per point."""
+    from paper_2602_05885_b200 import binding as B
+    from paper_2602_05885_b200 import workload
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks = measured_peaks()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    idx = 0
+    for H in (4096, 5120):
+        for V in (32768, 151936):
+            for T in (4096, 8192, 16384, 32768, 65536):
+                wl = workload.build("sweep", dev, seed=4000 + idx, sweep_shape=(T, V, H))
+                idx += 1
+                S = wl.S
+                g = torch.Generator(device=dev).manual_seed(idx)
+                seg_adv = torch.randn(S, generator=g, device=dev)
+                row = {"sweep_point": {"T": T, "V": V, "H": H}, "unit": UNIT}
+                for mode in ("wide", "off"):
+                    p = B.drk_pg_params_default()
+                    if mode == "wide":
+                        p.mrs_lo, p.mrs_hi = wl.wide_band()
+                    else:
+                        p.mrs_lo, p.mrs_hi, p.veto_ratio = 0.0, float("inf"), 0.0
+                    p.dh_dtype = B.DRK_BF16
+                    bufs = B.PgLossBuffers(T, H, V, S, B.DRK_BF16, p, dev)
+
+                    def call():
+                        B.drk_pg_loss_fwd_bwd(wl.hidden, wl.W, B.DRK_BF16, wl.ids, wl.rollout_logp, wl.loss_mask, wl.cu,
+                                              seg_adv, T, H, V, S, p, bufs.loss, bufs.logp, bufs.lse, bufs.seg_w,
+                                              bufs.seg_keep, bufs.counters, bufs.dH, bufs.dW, bufs.workspace,
+                                              bufs.workspace_bytes, bufs.status)
+                    for _ in range(3):
+                        call()
+                    torch.cuda.synchronize()
+                    e0.record()
+                    for _ in range(args.steps):
+                        call()
+                    e1.record()
+                    torch.cuda.synchronize()
+                    ms = e0.elapsed_time(e1) / args.steps
+                    Tc = int(bufs.counters[0].item())     # advantages are non-zero here: kept tokens = backward rows
+                    tf = (2.0 * T + 6.0 * Tc) * H * V / (ms * 1e-3) / 1e12
+                    row[mode] = {"ms": ms, "tokens_per_s": T / (ms * 1e-3), "rows_in_backward": Tc, "tflops": tf,
+                                 "frac_of_measured_sustained": tf / peaks["tflops"], "frac_of_nominal_2250": tf / 2250.0,
+                                 "status": int(bufs.status.item())}
+                    del bufs
+                print(json.dumps(row), flush=True)
+                del wl
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -172,11 +223,15 @@ def main():
     ap.add_argument("--cpu-tokens", type=int, default=512)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="roofline sweep over T x V x H instead of the headline run")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.sweep:
+        run_sweep(args)
         return
 
     from paper_2602_05885_b200 import binding as B

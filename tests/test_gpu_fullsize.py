@@ -129,14 +129,18 @@ def test_full_size_structured_rows():
     assert err <= Hh.TOL_GRAD_FRO, f"dW rel Frobenius err {err}"
 
 
-def test_full_size_bench_inputs_sampled_rows():
+@pytest.mark.parametrize("shape", [None, (4096, 32768, 4096), (65536, 151936, 5120)],
+                         ids=["bench-14b", "sweep-smallest", "sweep-largest"])
+def test_full_size_bench_inputs_sampled_rows(shape):
+    """The benchmark's own 14B-shaped micro-batch, and the smallest and largest points of the roofline sweep."""
     dev = torch.device("cuda:0")
-    wl = workload.build("qwen3-14b", dev, seed=2000)
+    wl = workload.build("qwen3-14b", dev, seed=2000) if shape is None else \
+        workload.build("sweep", dev, seed=4000, sweep_shape=shape)
     T, H, V, S = wl.T, wl.H, wl.V, wl.S
     # MRS off and an explicit scale: every coefficient is then known without the other rows' log-probs
     p = _bench_params(wl, mrs="off")
     p.norm = B.DRK_NORM_EXPLICIT
-    p.explicit_scale = F32(1.0 / 32768)
+    p.explicit_scale = F32(1.0 / T)
     g = torch.Generator().manual_seed(8)
     seg_adv = torch.randn(S, generator=g).float()
     bufs = _run(wl, p, seg_adv.to(dev))
