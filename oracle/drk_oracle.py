@@ -304,3 +304,74 @@ def pg_loss_fwd_bwd(hidden, W, ids, rollout_logp, loss_mask, cu_seqlens, seg_adv
         out["dH"] = dH
         out["dW"] = dW
     return out
+
+
+# ---------------------------------------------------------------------------
+# Reward front-end (Sec. 4.2 Eq. 1; Sec. 5.2 profiling-based reward and rejection sampling)
+# ---------------------------------------------------------------------------
+
+def speedup_reward(correct, t_ref, t_kernel, pr=None, clip=3.0):
+    """Eq. 1: R = C + C * min(T_ref / T_kernel, clip).  With a profiling ratio (Sec. 5.2) the
+    reward of a correct kernel additionally gains PR = T_generated / T_total."""
+    C = np.asarray(correct).astype(bool)
+    speed = np.minimum(np.asarray(t_ref, dtype=F64) / np.asarray(t_kernel, dtype=F64), float(clip))
+    R = np.where(C, 1.0 + speed, 0.0)
+    if pr is not None:
+        R = R + np.where(C, np.asarray(pr, dtype=F64), 0.0)
+    return R
+
+
+def prs_keep_prob(pr, tau=0.3, s=0.1):
+    """Sec. 5.2: p = clip((PR - tau) / s, 0, 1).  Taken in float32 (subtract, divide, clamp), the
+    precision in which the retention decision is made."""
+    pr32 = np.asarray(pr, dtype=np.float32)
+    p = (pr32 - np.float32(tau)) / np.float32(s)
+    return np.minimum(np.maximum(p, np.float32(0.0)), np.float32(1.0)).astype(np.float32)
+
+
+_PHILOX_M0, _PHILOX_M1 = 0xD2511F53, 0xCD9E8D57
+_PHILOX_W0, _PHILOX_W1 = 0x9E3779B9, 0xBB67AE85
+_MASK32 = 0xFFFFFFFF
+
+
+def philox4x32_10(counter, key):
+    """Philox-4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as
+    1, 2, 3", SC'11), written from its definition with Python integers."""
+    c0, c1, c2, c3 = [int(x) & _MASK32 for x in counter]
+    k0, k1 = [int(x) & _MASK32 for x in key]
+    for r in range(10):
+        if r > 0:
+            k0 = (k0 + _PHILOX_W0) & _MASK32
+            k1 = (k1 + _PHILOX_W1) & _MASK32
+        p0 = _PHILOX_M0 * c0
+        p1 = _PHILOX_M1 * c2
+        hi0, lo0 = p0 >> 32, p0 & _MASK32
+        hi1, lo1 = p1 >> 32, p1 & _MASK32
+        c0, c1, c2, c3 = (hi1 ^ c1 ^ k0) & _MASK32, lo1, (hi0 ^ c3 ^ k1) & _MASK32, lo0
+    return c0, c1, c2, c3
+
+
+def prs_uniform(seed, offset, index):
+    """The uniform in [0,1) that decides sample `index`: the top 24 bits of the first output word
+    of Philox-4x32-10 with key = seed (low, high word) and counter = (index, offset) (low, high
+    words each), scaled by 2^-24 (exact in float32)."""
+    x0 = philox4x32_10((index & _MASK32, (index >> 32) & _MASK32, offset & _MASK32, (offset >> 32) & _MASK32),
+                       (seed & _MASK32, (seed >> 32) & _MASK32))[0]
+    return np.float32((x0 >> 8) * (1.0 / 16777216.0))
+
+
+PRS_OFF, PRS_SOFT, PRS_HARD = 0, 1, 2
+
+
+def prs_retain(pr, tau=0.3, s=0.1, mode=PRS_SOFT, seed=0, offset=0):
+    """Profiling-based rejection sampling: sample i is retained with probability p_i (soft), or iff
+    PR_i >= tau (the hard-threshold variant of the PRS ablation, App. D), or always (off)."""
+    pr = np.asarray(pr, dtype=np.float32)
+    n = pr.shape[0]
+    if mode == PRS_OFF:
+        return np.ones(n, dtype=bool)
+    if mode == PRS_HARD:
+        return pr >= np.float32(tau)
+    p = prs_keep_prob(pr, tau, s)
+    u = np.array([prs_uniform(seed, offset, i) for i in range(n)], dtype=np.float32)
+    return u < p
