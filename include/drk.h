@@ -81,6 +81,39 @@ int drk_trloo_advantage(const float* reward, const uint8_t* valid,
                         float gamma, int32_t baseline, float* ret, float* adv,
                         int32_t* gsize, void* stream);
 
+/*
+ * Reward front-end, upstream of drk_trloo_advantage: per-sample reward and the retention decision of
+ * profiling-based rejection sampling.
+ *
+ *   speedup = min(t_ref / t_kernel, speedup_clip)                      (Sec. 4.2, clip 3)
+ *   reward  = C + C * speedup (+ C * PR when use_pr)                    (Eq. 1; profiling reward of Sec. 5.2)
+ *   p       = clip((PR - prs_tau) / prs_s, 0, 1)                        (Sec. 5.2, tau = 0.3, s = 0.1)
+ *   retain  = 1                          prs_mode = DRK_PRS_OFF
+ *             u < p, u ~ U[0,1)          prs_mode = DRK_PRS_SOFT
+ *             PR >= prs_tau              prs_mode = DRK_PRS_HARD        (ablation without softness, App. D)
+ *
+ * u is the top 24 bits, times 2^-24, of the first output word of Philox-4x32-10 (Salmon et al., SC'11)
+ * with key = seed (low, high word) and counter = (sample index, offset) (low, high word each): the draw
+ * for sample i depends on (seed, offset, i) only.  p and the comparison are taken in fp32.
+ * correct [n] uint8 (C = correct != 0), t_ref, t_kernel, pr [n] float, reward [n] float, retain [n] uint8:
+ * device.  pr may be NULL when use_pr = 0 and prs_mode = DRK_PRS_OFF; retain may be NULL when
+ * prs_mode = DRK_PRS_OFF.  A rejected sample is one the caller leaves out of the loss (clear its
+ * loss-mask tokens or give it zero advantage); its reward still enters the group baseline.
+ */
+typedef enum { DRK_PRS_OFF = 0, DRK_PRS_SOFT = 1, DRK_PRS_HARD = 2 } drk_prs_mode;
+typedef struct {
+  float speedup_clip; /* default 3 */
+  int32_t use_pr;     /* default 0 */
+  int32_t prs_mode;   /* drk_prs_mode, default DRK_PRS_OFF */
+  float prs_tau;      /* default 0.3 */
+  float prs_s;        /* default 0.1 */
+  uint64_t seed;      /* default 0 */
+  uint64_t offset;    /* default 0; advance per call to draw fresh numbers with one seed */
+} drk_reward_params;
+void drk_reward_params_default(drk_reward_params* p); /* host pointer */
+int drk_reward(const uint8_t* correct, const float* t_ref, const float* t_kernel, const float* pr, int64_t n,
+               const drk_reward_params* p, float* reward, uint8_t* retain, void* stream);
+
 /* Parameters of the fused loss.  Fill with drk_pg_params_default() first. */
 typedef struct {
   float mrs_lo;          /* Sec. 5.1: retain a sample iff mrs_lo <= w <= mrs_hi; default 0.999       */

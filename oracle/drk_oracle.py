@@ -375,3 +375,45 @@ def prs_retain(pr, tau=0.3, s=0.1, mode=PRS_SOFT, seed=0, offset=0):
     p = prs_keep_prob(pr, tau, s)
     u = np.array([prs_uniform(seed, offset, i) for i in range(n)], dtype=np.float32)
     return u < p
+
+
+# ---------------------------------------------------------------------------
+# Stability diagnostics (the quantities monitored in Sec. 5.1 / App. B: entropy, perplexities of the
+# trainer and of the rollout engine, log-ratio statistics, gradient norms)
+# ---------------------------------------------------------------------------
+
+def token_entropy(s):
+    """Entropy of softmax(s[t,:]) per row: H_t = -sum_v p_v ln p_v = lse_t - sum_v p_v s_v."""
+    lse = logsumexp_rows(s)
+    p = np.exp(s - lse[:, None])
+    return lse - np.sum(p * s, axis=1)
+
+
+def diagnostics(logp, rollout_logp, entropy, loss_mask, cu_seqlens, dH=None, dW=None):
+    """Means over the loss-masked tokens that lie inside segments.  Returns a dict:
+    n_tokens, mean_entropy, ppl_train = exp(-mean logp), ppl_rollout = exp(-mean rollout_logp),
+    mean_log_ratio = mean(logp - rollout_logp), max_abs_log_ratio, grad_norm_dH, grad_norm_dW
+    (Frobenius norms; 0 when the gradient is not given)."""
+    logp = np.asarray(logp, dtype=F64)
+    rl = np.asarray(rollout_logp, dtype=F64)
+    mask = np.asarray(loss_mask).astype(bool)
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    sel = np.zeros(logp.shape[0], dtype=bool)
+    for g in range(cu.shape[0] - 1):
+        sel[cu[g]:cu[g + 1]] = True
+    sel &= mask
+    n = int(sel.sum())
+    out = dict(n_tokens=n, mean_entropy=0.0, ppl_train=1.0, ppl_rollout=1.0, mean_log_ratio=0.0,
+               max_abs_log_ratio=0.0, grad_norm_dH=0.0, grad_norm_dW=0.0)
+    if n > 0:
+        d = logp[sel] - rl[sel]
+        out["mean_entropy"] = float(np.asarray(entropy, dtype=F64)[sel].sum() / n) if entropy is not None else 0.0
+        out["ppl_train"] = math.exp(-float(logp[sel].sum()) / n)
+        out["ppl_rollout"] = math.exp(-float(rl[sel].sum()) / n)
+        out["mean_log_ratio"] = float(d.sum() / n)
+        out["max_abs_log_ratio"] = float(np.abs(d).max())
+    if dH is not None:
+        out["grad_norm_dH"] = float(np.sqrt(np.sum(np.asarray(dH, dtype=F64) ** 2)))
+    if dW is not None:
+        out["grad_norm_dW"] = float(np.sqrt(np.sum(np.asarray(dW, dtype=F64) ** 2)))
+    return out

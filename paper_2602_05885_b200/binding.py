@@ -54,6 +54,21 @@ class drk_pg_params(ctypes.Structure):
     ]
 
 
+class drk_reward_params(ctypes.Structure):
+    _fields_ = [
+        ("speedup_clip", ctypes.c_float),
+        ("use_pr", ctypes.c_int32),
+        ("prs_mode", ctypes.c_int32),
+        ("prs_tau", ctypes.c_float),
+        ("prs_s", ctypes.c_float),
+        ("seed", ctypes.c_uint64),
+        ("offset", ctypes.c_uint64),
+    ]
+
+
+DRK_PRS_OFF, DRK_PRS_SOFT, DRK_PRS_HARD = 0, 1, 2
+
+
 class DrkError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
@@ -87,6 +102,10 @@ def load() -> ctypes.CDLL:
     lib.drk_trloo_advantage.restype = ctypes.c_int
     lib.drk_pg_logprob_fwd.argtypes = [vp, vp, i32, vp, i64, i32, i32, i32, vp, vp, vp, sz, vp, vp]
     lib.drk_pg_logprob_fwd.restype = ctypes.c_int
+    lib.drk_reward_params_default.argtypes = [ctypes.POINTER(drk_reward_params)]
+    lib.drk_reward_params_default.restype = None
+    lib.drk_reward.argtypes = [vp, vp, vp, vp, i64, ctypes.POINTER(drk_reward_params), vp, vp, vp]
+    lib.drk_reward.restype = ctypes.c_int
     lib.drk_pg_logprob_fwd_noalloc.argtypes = [vp, vp, i32, vp, i64, i32, i32, i32, vp, vp, vp, vp]
     lib.drk_pg_logprob_fwd_noalloc.restype = ctypes.c_int
     lib.drk_pg_loss_fwd_bwd.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, i64, i32, i32, i32,
@@ -149,6 +168,21 @@ def drk_pg_params_default() -> drk_pg_params:
 def drk_pg_workspace_bytes(T: int, H: int, V: int, S: int, in_dtype: int,
                            p: Optional[drk_pg_params], which: int) -> int:
     return int(load().drk_pg_workspace_bytes(T, H, V, S, in_dtype, ctypes.byref(p) if p is not None else None, which))
+
+
+def drk_reward_params_default() -> drk_reward_params:
+    p = drk_reward_params()
+    load().drk_reward_params_default(ctypes.byref(p))
+    return p
+
+
+def drk_reward(correct, t_ref, t_kernel, pr, n: int, p: Optional[drk_reward_params], reward, retain, stream=None,
+               check: bool = True) -> int:
+    rc = load().drk_reward(_ptr(correct), _ptr(t_ref), _ptr(t_kernel), _ptr(pr), n,
+                           ctypes.byref(p) if p is not None else None, _ptr(reward), _ptr(retain), _stream(stream))
+    if check and rc != DRK_OK:
+        raise DrkError(rc, "drk_reward")
+    return rc
 
 
 def drk_trloo_advantage(reward, valid, prompt_of_rollout, R: int, Tmax: int, gamma: float, baseline: int,
