@@ -183,7 +183,7 @@ def run_sweep(args):
 
                     def call():
                         B.drk_pg_loss_fwd_bwd(wl.hidden, wl.W, B.DRK_BF16, wl.ids, wl.rollout_logp, wl.loss_mask, wl.cu,
-                                              seg_adv, T, H, V, S, p, bufs.loss, bufs.logp, bufs.lse, bufs.seg_w,
+                                              seg_adv, T, H, V, S, p, bufs.loss, bufs.logp, bufs.lse, None, bufs.seg_w,
                                               bufs.seg_keep, bufs.counters, bufs.dH, bufs.dW, bufs.workspace,
                                               bufs.workspace_bytes, bufs.status)
                     for _ in range(3):
@@ -277,7 +277,7 @@ def main():
         launches[0] += B.drk_last_launch_count()
         seg_adv = adv.view(-1).index_select(0, seg_flat)     # the caller's gather of per-sample advantages
         B.drk_pg_loss_fwd_bwd(hidden, wl.W, code, ids, rl, mask, cu, seg_adv, T, H, V, S, p, bufs.loss, bufs.logp,
-                              bufs.lse, bufs.seg_w, bufs.seg_keep, bufs.counters, bufs.dH, bufs.dW,
+                              bufs.lse, bufs.entropy, bufs.seg_w, bufs.seg_keep, bufs.counters, bufs.dH, bufs.dW,
                               bufs.workspace, bufs.workspace_bytes, bufs.status, stream)
         launches[0] += B.drk_last_launch_count()
 
@@ -318,7 +318,7 @@ def main():
         for _ in range(reps):
             e0.record(stream)
             B.drk_pg_loss_fwd_bwd(wl.hidden, wl.W, code, wl.ids, wl.rollout_logp, wl.loss_mask, wl.cu, seg_adv, T, H,
-                                  V, S, pp, bufs.loss, bufs.logp, bufs.lse, bufs.seg_w, bufs.seg_keep, bufs.counters,
+                                  V, S, pp, bufs.loss, bufs.logp, bufs.lse, bufs.entropy, bufs.seg_w, bufs.seg_keep, bufs.counters,
                                   bufs.dH, bufs.dW, bufs.workspace, bufs.workspace_bytes, bufs.status, stream)
             e1.record(stream)
             torch.cuda.synchronize()

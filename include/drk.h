@@ -127,6 +127,11 @@ typedef struct {
   int32_t engine;        /* drk_engine; default DRK_ENGINE_AUTO                                      */
   int32_t v_chunk;       /* vocabulary columns whose dLogits are held at once in the backward;
                             0 = library default; rounded up to a multiple of 256                    */
+  int32_t keep_from_caller; /* 0: seg_keep is an output, decided by MRS here.  1: seg_keep is an INPUT:
+                            the caller has already decided which samples are retained (e.g. a sample
+                            split over several micro-batches, judged on log-probs from
+                            drk_pg_logprob_fwd of all its pieces); seg_w and the counters are still
+                            computed from this micro-batch's tokens                                   */
 } drk_pg_params;
 
 void drk_pg_params_default(drk_pg_params* p); /* host pointer */
@@ -150,13 +155,16 @@ size_t drk_pg_workspace_bytes(int64_t T, int32_t H, int32_t V, int32_t S, int32_
  *
  * hidden [T,H], W [V,H]: device, dtype in_dtype (both the same), 16-byte
  * aligned; for DRK_BF16, H must be a multiple of 8.  ids [T] int32 device.
- * logp, lse [T] float device.  status: device uint32, OR-ed into (the caller
- * zeroes it).  engine: drk_engine.  T = 0 enqueues nothing.  T <= 2^24,
- * 1 <= V <= 2^24, 1 <= H <= 65536.
+ * logp, lse [T] float device.  entropy: [T] float device or NULL; when given it
+ * receives the entropy of row t's distribution, lse[t] - sum_v p[t,v] s[t,v]
+ * (one of the quantities monitored in Sec. 5.1), from the same pass.  status:
+ * device uint32, OR-ed into (the caller zeroes it).  engine: drk_engine.
+ * T = 0 enqueues nothing.  T <= 2^24, 1 <= V <= 2^24, 1 <= H <= 65536.
  */
 int drk_pg_logprob_fwd(const void* hidden, const void* W, int32_t in_dtype, const int32_t* ids,
                        int64_t T, int32_t H, int32_t V, int32_t engine, float* logp, float* lse,
-                       void* workspace, size_t workspace_bytes, uint32_t* status, void* stream);
+                       float* entropy, void* workspace, size_t workspace_bytes, uint32_t* status,
+                       void* stream);
 
 /*
  * The same computation as drk_pg_logprob_fwd for callers that cannot hand over a workspace because they
@@ -166,8 +174,8 @@ int drk_pg_logprob_fwd(const void* hidden, const void* W, int32_t in_dtype, cons
  * packaging variant of the forward call above.)  The scratch (per-row partial max / sum-exp pairs and
  * target logits) lives in a fixed array inside the library image instead:
  *   - every GPU on which the library is loaded holds DRK_NOALLOC_SCRATCH_BYTES until the process exits;
- *   - if the sizes need more (roughly 8*nsplit*T + 4*T bytes, nsplit <= 32 chosen from T and V) the call
- *     returns DRK_ERR_WORKSPACE and enqueues nothing; T = 32768 at V = 151936 needs about 1.2 MB;
+ *   - if the sizes need more (roughly 16*nsplit*T + 4*T bytes, nsplit <= 32 chosen from T, H and V) the call
+ *     returns DRK_ERR_WORKSPACE and enqueues nothing; T = 32768 at H = 5120, V = 151936 needs about 2.2 MB;
  *   - the array is shared by all calls on a device and keeps the last call's contents.  What the
  *     computation reads is rewritten or cleared by each call, so consecutive calls on one stream are
  *     independent; calls that may run concurrently on the GPU (unordered streams) race on it;
@@ -199,7 +207,8 @@ int drk_pg_logprob_fwd_noalloc(const void* hidden, const void* W, int32_t in_dty
  *
  * rollout_logp [T] float, loss_mask [T] uint8, cu_seqlens [S+1] int32
  * (non-decreasing, within [0,T]), seg_adv [S] float: device.  Outputs, all
- * device: loss [1] float; logp, lse [T]; seg_w [S] float; seg_keep [S] uint8;
+ * device: loss [1] float; logp, lse [T]; entropy [T] or NULL (as in the forward
+ * call); seg_w [S] float; seg_keep [S] uint8;
  * counters [4] int64 = {kept masked tokens, masked tokens in segments, kept
  * segments, vetoed segments}; dH [T,H] of p->dh_dtype; dW [V,H] of
  * p->dw_dtype.  dH and dW must be 16-byte aligned.  With bf16 inputs dL is
@@ -211,9 +220,24 @@ int drk_pg_loss_fwd_bwd(const void* hidden, const void* W, int32_t in_dtype, con
                         const float* rollout_logp, const uint8_t* loss_mask,
                         const int32_t* cu_seqlens, const float* seg_adv, int64_t T, int32_t H,
                         int32_t V, int32_t S, const drk_pg_params* p, float* loss, float* logp,
-                        float* lse, float* seg_w, uint8_t* seg_keep, int64_t* counters, void* dH,
-                        void* dW, void* workspace, size_t workspace_bytes, uint32_t* status,
+                        float* lse, float* entropy, float* seg_w, uint8_t* seg_keep, int64_t* counters,
+                        void* dH, void* dW, void* workspace, size_t workspace_bytes, uint32_t* status,
                         void* stream);
+
+/*
+ * Stability diagnostics of one micro-batch, from the outputs of the calls above: what the paper
+ * monitors to diagnose training / inference mismatch (Sec. 5.1, App. B: entropy, perplexity of the
+ * trainer and of the rollout engine, gradient norm).  Means run over the loss-masked tokens inside
+ * segments.  out: device double[8] =
+ *   { n_tokens, mean entropy, exp(-mean logp), exp(-mean rollout_logp), mean (logp - rollout_logp),
+ *     max |logp - rollout_logp|, ||dH||_F, ||dW||_F }.
+ * entropy, dH, dW may be NULL (their entries are then 0).  dH is [T,H], dW is [V,H] of the given
+ * dtypes.  Sums use fp64 atomics: the last digits are not reproducible bit for bit.
+ */
+int drk_pg_diagnostics(const float* logp, const float* rollout_logp, const float* entropy,
+                       const uint8_t* loss_mask, const int32_t* cu_seqlens, int64_t T, int32_t S,
+                       const void* dH, int32_t dh_dtype, const void* dW, int32_t dw_dtype, int32_t H,
+                       int32_t V, double* out, void* stream);
 
 /* Number of kernels the last call on this host thread enqueued (0 after an error). */
 int drk_last_launch_count(void);

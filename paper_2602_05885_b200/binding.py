@@ -51,6 +51,7 @@ class drk_pg_params(ctypes.Structure):
         ("dw_accumulate", ctypes.c_int32),
         ("engine", ctypes.c_int32),
         ("v_chunk", ctypes.c_int32),
+        ("keep_from_caller", ctypes.c_int32),
     ]
 
 
@@ -100,7 +101,7 @@ def load() -> ctypes.CDLL:
     lib.drk_pg_workspace_bytes.restype = sz
     lib.drk_trloo_advantage.argtypes = [vp, vp, vp, i32, i32, f32, i32, vp, vp, vp, vp]
     lib.drk_trloo_advantage.restype = ctypes.c_int
-    lib.drk_pg_logprob_fwd.argtypes = [vp, vp, i32, vp, i64, i32, i32, i32, vp, vp, vp, sz, vp, vp]
+    lib.drk_pg_logprob_fwd.argtypes = [vp, vp, i32, vp, i64, i32, i32, i32, vp, vp, vp, vp, sz, vp, vp]
     lib.drk_pg_logprob_fwd.restype = ctypes.c_int
     lib.drk_reward_params_default.argtypes = [ctypes.POINTER(drk_reward_params)]
     lib.drk_reward_params_default.restype = None
@@ -109,8 +110,10 @@ def load() -> ctypes.CDLL:
     lib.drk_pg_logprob_fwd_noalloc.argtypes = [vp, vp, i32, vp, i64, i32, i32, i32, vp, vp, vp, vp]
     lib.drk_pg_logprob_fwd_noalloc.restype = ctypes.c_int
     lib.drk_pg_loss_fwd_bwd.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, i64, i32, i32, i32,
-                                        ctypes.POINTER(drk_pg_params), vp, vp, vp, vp, vp, vp, vp, vp, vp, sz,
+                                        ctypes.POINTER(drk_pg_params), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz,
                                         vp, vp]
+    lib.drk_pg_diagnostics.argtypes = [vp, vp, vp, vp, vp, i64, i32, vp, i32, vp, i32, i32, i32, vp, vp]
+    lib.drk_pg_diagnostics.restype = ctypes.c_int
     lib.drk_pg_loss_fwd_bwd.restype = ctypes.c_int
     lib.drk_last_launch_count.argtypes = []
     lib.drk_last_launch_count.restype = ctypes.c_int
@@ -194,10 +197,10 @@ def drk_trloo_advantage(reward, valid, prompt_of_rollout, R: int, Tmax: int, gam
     return rc
 
 
-def drk_pg_logprob_fwd(hidden, W, in_dtype: int, ids, T: int, H: int, V: int, engine: int, logp, lse,
+def drk_pg_logprob_fwd(hidden, W, in_dtype: int, ids, T: int, H: int, V: int, engine: int, logp, lse, entropy,
                        workspace, workspace_bytes: int, status, stream=None, check: bool = True) -> int:
     rc = load().drk_pg_logprob_fwd(_ptr(hidden), _ptr(W), in_dtype, _ptr(ids), T, H, V, engine, _ptr(logp), _ptr(lse),
-                                   _ptr(workspace), workspace_bytes, _ptr(status), _stream(stream))
+                                   _ptr(entropy), _ptr(workspace), workspace_bytes, _ptr(status), _stream(stream))
     if check and rc != DRK_OK:
         raise DrkError(rc, "drk_pg_logprob_fwd")
     return rc
@@ -220,17 +223,30 @@ def drk_pg_logprob_fwd_noalloc(hidden, W, in_dtype: int, ids, T: int, H: int, V:
 
 
 def drk_pg_loss_fwd_bwd(hidden, W, in_dtype: int, ids, rollout_logp, loss_mask, cu_seqlens, seg_adv,
-                        T: int, H: int, V: int, S: int, p: Optional[drk_pg_params], loss, logp, lse, seg_w,
-                        seg_keep, counters, dH, dW, workspace, workspace_bytes: int, status, stream=None,
+                        T: int, H: int, V: int, S: int, p: Optional[drk_pg_params], loss, logp, lse, entropy,
+                        seg_w, seg_keep, counters, dH, dW, workspace, workspace_bytes: int, status, stream=None,
                         check: bool = True) -> int:
     rc = load().drk_pg_loss_fwd_bwd(_ptr(hidden), _ptr(W), in_dtype, _ptr(ids), _ptr(rollout_logp), _ptr(loss_mask),
                                     _ptr(cu_seqlens), _ptr(seg_adv), T, H, V, S,
                                     ctypes.byref(p) if p is not None else None, _ptr(loss), _ptr(logp), _ptr(lse),
-                                    _ptr(seg_w), _ptr(seg_keep), _ptr(counters), _ptr(dH), _ptr(dW),
+                                    _ptr(entropy), _ptr(seg_w), _ptr(seg_keep), _ptr(counters), _ptr(dH), _ptr(dW),
                                     _ptr(workspace), workspace_bytes, _ptr(status), _stream(stream))
     if check and rc != DRK_OK:
         raise DrkError(rc, "drk_pg_loss_fwd_bwd")
     return rc
+
+
+def drk_pg_diagnostics(logp, rollout_logp, entropy, loss_mask, cu_seqlens, T: int, S: int, dH, dh_dtype: int,
+                       dW, dw_dtype: int, H: int, V: int, out, stream=None, check: bool = True) -> int:
+    rc = load().drk_pg_diagnostics(_ptr(logp), _ptr(rollout_logp), _ptr(entropy), _ptr(loss_mask), _ptr(cu_seqlens),
+                                   T, S, _ptr(dH), dh_dtype, _ptr(dW), dw_dtype, H, V, _ptr(out), _stream(stream))
+    if check and rc != DRK_OK:
+        raise DrkError(rc, "drk_pg_diagnostics")
+    return rc
+
+
+DIAG_FIELDS = ("n_tokens", "mean_entropy", "ppl_train", "ppl_rollout", "mean_log_ratio", "max_abs_log_ratio",
+               "grad_norm_dH", "grad_norm_dW")
 
 
 # ---------------------------------------------------------------------------
@@ -253,7 +269,8 @@ def trloo_advantage(reward: torch.Tensor, valid: torch.Tensor, prompt_of_rollout
     return ret, adv, gsize
 
 
-def pg_logprob_fwd(hidden: torch.Tensor, W: torch.Tensor, ids: torch.Tensor, engine: int = DRK_ENGINE_AUTO):
+def pg_logprob_fwd(hidden: torch.Tensor, W: torch.Tensor, ids: torch.Tensor, engine: int = DRK_ENGINE_AUTO,
+                   entropy: Optional[torch.Tensor] = None):
     T, H = hidden.shape
     V = W.shape[0]
     code = _dtype_code(hidden)
@@ -264,7 +281,7 @@ def pg_logprob_fwd(hidden: torch.Tensor, W: torch.Tensor, ids: torch.Tensor, eng
     logp = torch.empty(T, dtype=torch.float32, device=hidden.device)
     lse = torch.empty(T, dtype=torch.float32, device=hidden.device)
     status = torch.zeros(1, dtype=torch.int32, device=hidden.device)
-    drk_pg_logprob_fwd(hidden, W, code, ids, T, H, V, engine, logp, lse, ws, nbytes, status)
+    drk_pg_logprob_fwd(hidden, W, code, ids, T, H, V, engine, logp, lse, entropy, ws, nbytes, status)
     return logp, lse, status
 
 
@@ -278,6 +295,7 @@ class PgLossBuffers:
         self.loss = torch.zeros(1, **f32)
         self.logp = torch.empty(T, **f32)
         self.lse = torch.empty(T, **f32)
+        self.entropy = torch.empty(T, **f32)
         self.seg_w = torch.empty(S, **f32)
         self.seg_keep = torch.empty(S, dtype=torch.uint8, device=device)
         self.counters = torch.zeros(4, dtype=torch.int64, device=device)
@@ -301,6 +319,7 @@ def pg_loss_fwd_bwd(hidden, W, ids, rollout_logp, loss_mask, cu_seqlens, seg_adv
     if bufs is None:
         bufs = PgLossBuffers(T, H, V, S, code, p, hidden.device)
     drk_pg_loss_fwd_bwd(hidden, W, code, ids, rollout_logp, loss_mask, cu_seqlens, seg_adv, T, H, V, S, p,
-                        bufs.loss, bufs.logp, bufs.lse, bufs.seg_w, bufs.seg_keep, bufs.counters, bufs.dH, bufs.dW,
+                        bufs.loss, bufs.logp, bufs.lse, bufs.entropy, bufs.seg_w, bufs.seg_keep, bufs.counters, bufs.dH,
+                        bufs.dW,
                         bufs.workspace, bufs.workspace_bytes, bufs.status, stream)
     return bufs

@@ -84,7 +84,7 @@ struct FwdWs {
 FwdWs carve_fwd(Carver& c, int64_t T, int V, bool simt, int engine) {
   FwdWs w;
   w.nsplit = simt ? simt_nsplit(T, V) : umma_nsplit(T, V, umma_ctas(engine));
-  w.part = static_cast<float*>(c.take(sizeof(float) * 2 * (size_t)w.nsplit * (size_t)T));
+  w.part = static_cast<float*>(c.take(sizeof(float) * 4 * (size_t)w.nsplit * (size_t)T));
   w.tgt = static_cast<float*>(c.take(sizeof(float) * (size_t)T));
   return w;
 }
@@ -129,18 +129,20 @@ bool params_ok(const drk_pg_params& p) {
   if (p.dh_dtype != DRK_F32 && p.dh_dtype != DRK_BF16) return false;
   if (!engine_ok(p.engine)) return false;
   if (p.v_chunk < 0) return false;
+  if (p.keep_from_caller != 0 && p.keep_from_caller != 1) return false;
   if (std::isnan(p.mrs_lo) || std::isnan(p.mrs_hi) || std::isnan(p.veto_ratio)) return false;
   if (p.norm == DRK_NORM_EXPLICIT && !std::isfinite(p.explicit_scale)) return false;
   return true;
 }
 
 int run_fwd(const void* hidden, const void* W, int in_dtype, const int32_t* ids, int64_t T, int H, int V,
-            bool simt, int engine, const FwdWs& w, float* logp, float* lse, uint32_t* status, cudaStream_t st) {
+            bool simt, int engine, const FwdWs& w, float* logp, float* lse, float* entropy, uint32_t* status,
+            cudaStream_t st) {
   if (simt) {
-    SimtFwdArgs a{hidden, W, in_dtype, ids, T, H, V, logp, lse, w.part, w.tgt, w.nsplit, status};
+    SimtFwdArgs a{hidden, W, in_dtype, ids, T, H, V, logp, lse, w.part, w.tgt, w.nsplit, status, entropy};
     return launch_simt_fwd(a, st);
   }
-  UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, w.part, w.tgt, w.nsplit, status, umma_ctas(engine)};
+  UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, w.part, w.tgt, w.nsplit, status, umma_ctas(engine), entropy};
   return launch_umma_fwd(a, st);
 }
 
@@ -163,6 +165,7 @@ void drk_pg_params_default(drk_pg_params* p) {
   p->dw_accumulate = 0;
   p->engine = DRK_ENGINE_AUTO;
   p->v_chunk = 0;
+  p->keep_from_caller = 0;
 }
 
 size_t drk_pg_workspace_bytes(int64_t T, int32_t H, int32_t V, int32_t S, int32_t in_dtype,
@@ -196,7 +199,7 @@ int drk_trloo_advantage(const float* reward, const uint8_t* valid, const int32_t
 }
 
 int drk_pg_logprob_fwd(const void* hidden, const void* W, int32_t in_dtype, const int32_t* ids, int64_t T,
-                       int32_t H, int32_t V, int32_t engine, float* logp, float* lse, void* workspace,
+                       int32_t H, int32_t V, int32_t engine, float* logp, float* lse, float* entropy, void* workspace,
                        size_t workspace_bytes, uint32_t* status, void* stream) {
   g_launches = 0;
   if (!sizes_ok(T, H, V, in_dtype)) return DRK_ERR_INVALID_ARG;
@@ -214,7 +217,8 @@ int drk_pg_logprob_fwd(const void* hidden, const void* W, int32_t in_dtype, cons
   if (rc != DRK_OK) return rc;
   Carver c(workspace);
   const FwdWs w = carve_fwd(c, T, V, simt, engine);
-  rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, engine, w, logp, lse, status, static_cast<cudaStream_t>(stream));
+  rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, engine, w, logp, lse, entropy, status,
+               static_cast<cudaStream_t>(stream));
   if (rc != DRK_OK) g_launches = 0;
   return rc;
 }
@@ -222,8 +226,8 @@ int drk_pg_logprob_fwd(const void* hidden, const void* W, int32_t in_dtype, cons
 int drk_pg_loss_fwd_bwd(const void* hidden, const void* W, int32_t in_dtype, const int32_t* ids,
                         const float* rollout_logp, const uint8_t* loss_mask, const int32_t* cu_seqlens,
                         const float* seg_adv, int64_t T, int32_t H, int32_t V, int32_t S, const drk_pg_params* pp,
-                        float* loss, float* logp, float* lse, float* seg_w, uint8_t* seg_keep, int64_t* counters,
-                        void* dH, void* dW, void* workspace, size_t workspace_bytes, uint32_t* status,
+                        float* loss, float* logp, float* lse, float* entropy, float* seg_w, uint8_t* seg_keep,
+                        int64_t* counters, void* dH, void* dW, void* workspace, size_t workspace_bytes, uint32_t* status,
                         void* stream) {
   g_launches = 0;
   drk_pg_params p;
@@ -249,7 +253,7 @@ int drk_pg_loss_fwd_bwd(const void* hidden, const void* W, int32_t in_dtype, con
   auto fail = [&](int code) { g_launches = 0; return code; };
 
   if (T > 0) {
-    rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, p.engine, fw, logp, lse, status, st);
+    rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, p.engine, fw, logp, lse, entropy, status, st);
     if (rc != DRK_OK) return fail(rc);
   }
   MrsArgs m{};
@@ -258,7 +262,7 @@ int drk_pg_loss_fwd_bwd(const void* hidden, const void* W, int32_t in_dtype, con
   m.ln_lo = p.mrs_lo > 0.f ? std::log((double)p.mrs_lo) : -std::numeric_limits<double>::infinity();
   m.ln_hi = std::isinf(p.mrs_hi) ? std::numeric_limits<double>::infinity() : std::log((double)p.mrs_hi);
   m.ln_veto = p.veto_ratio > 0.f ? std::log((double)p.veto_ratio) : -std::numeric_limits<double>::infinity();
-  m.norm = p.norm; m.explicit_scale = p.explicit_scale;
+  m.norm = p.norm; m.explicit_scale = p.explicit_scale; m.keep_from_caller = p.keep_from_caller;
   m.seg_w = seg_w; m.seg_keep = seg_keep; m.loss = loss; m.counters = counters; m.coeff = bw.coeff;
   m.seg_stats = bw.seg_stats; m.status = status;
   rc = launch_mrs(m, st);

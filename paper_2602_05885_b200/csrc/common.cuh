@@ -40,7 +40,7 @@ int launch_trloo(const float* reward, const uint8_t* valid, const int32_t* promp
 struct MrsArgs {
   const float* logp; const float* rollout_logp; const uint8_t* loss_mask; const int32_t* cu;
   const float* seg_adv; int64_t T; int S;
-  double ln_lo, ln_hi, ln_veto; int norm; float explicit_scale;
+  double ln_lo, ln_hi, ln_veto; int norm; float explicit_scale; int keep_from_caller;
   float* seg_w; uint8_t* seg_keep; float* loss; int64_t* counters; float* coeff /*[T]*/;
   double* seg_stats /*[S*4] workspace*/; uint32_t* status;
 };
@@ -49,12 +49,13 @@ int launch_mrs(const MrsArgs& a, cudaStream_t st);
 // FFMA path.
 struct SimtFwdArgs {
   const void* hidden; const void* W; int in_dtype; const int32_t* ids; int64_t T; int H; int V;
-  float* logp; float* lse; float* part /*[nsplit*T*2]*/; float* tgt /*[T]*/; int nsplit; uint32_t* status;
+  float* logp; float* lse; float* part /*[nsplit*T*4]*/; float* tgt /*[T]*/; int nsplit; uint32_t* status;
+  float* entropy /*[T] or null*/;
 };
 int simt_nsplit(int64_t T, int V);
 int launch_simt_fwd(const SimtFwdArgs& a, cudaStream_t st);
 int launch_lse_merge(const float* part, const float* tgt, const int32_t* ids, int64_t T, int V, int nsplit,
-                     float* logp, float* lse, uint32_t* status, cudaStream_t st);
+                     float* logp, float* lse, float* entropy, uint32_t* status, cudaStream_t st);
 struct SimtBwdArgs {
   const void* hidden; const void* W; int in_dtype; const int32_t* ids; int64_t T; int H; int V;
   const float* lse; const float* coeff; float* dL /*[T*vc] fp32 workspace*/; int vc;
@@ -66,8 +67,9 @@ int launch_simt_bwd(const SimtBwdArgs& a, cudaStream_t st);
 // tcgen05 path (bf16 inputs).
 struct UmmaFwdArgs {
   const void* hidden; const void* W; const int32_t* ids; int64_t T; int H; int V;
-  float* logp; float* lse; float* part /*[nsplit*T*2]*/; float* tgt; int nsplit; uint32_t* status;
+  float* logp; float* lse; float* part /*[nsplit*T*4]*/; float* tgt; int nsplit; uint32_t* status;
   int ctas /*1: one CTA per tile; 2: CTA pairs*/;
+  float* entropy /*[T] or null*/;
 };
 int umma_nsplit(int64_t T, int V, int ctas);
 int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st);

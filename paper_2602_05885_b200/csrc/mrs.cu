@@ -101,7 +101,8 @@ __device__ double block_sum(double x, double* sh) {
 
 __global__ void __launch_bounds__(kFinThreads)
 finalize_kernel(double* __restrict__ seg_stats, const float* __restrict__ seg_adv, int S, double ln_lo,
-                double ln_hi, double ln_veto, int norm, float explicit_scale, float* __restrict__ seg_w,
+                double ln_hi, double ln_veto, int norm, float explicit_scale, int keep_from_caller,
+                float* __restrict__ seg_w,
                 uint8_t* __restrict__ seg_keep, float* __restrict__ loss, int64_t* __restrict__ counters) {
   __shared__ double sh[kFinThreads];
   double kept_tok = 0, masked_tok = 0, kept_seg = 0, veto_seg = 0;
@@ -115,6 +116,7 @@ finalize_kernel(double* __restrict__ seg_stats, const float* __restrict__ seg_ad
       w = (float)exp(mean);
       vetoed = st[2] < ln_veto;
       keep = (ln_lo <= mean) && (mean <= ln_hi) && !vetoed;
+      if (keep_from_caller) keep = seg_keep[g] != 0;   // the caller's decision stands (never for empty segments)
     }
     seg_w[g] = w;
     seg_keep[g] = keep ? 1 : 0;
@@ -173,7 +175,7 @@ int launch_mrs(const MrsArgs& a, cudaStream_t st) {
                                                   a.seg_stats, a.status);
   DRK_LAUNCHED();
   finalize_kernel<<<1, kFinThreads, 0, st>>>(a.seg_stats, a.seg_adv, a.S, a.ln_lo, a.ln_hi,
-                                             a.ln_veto, a.norm, a.explicit_scale, a.seg_w,
+                                             a.ln_veto, a.norm, a.explicit_scale, a.keep_from_caller, a.seg_w,
                                              a.seg_keep, a.loss, a.counters);
   DRK_LAUNCHED();
   if (a.T > 0) {

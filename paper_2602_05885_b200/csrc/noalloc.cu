@@ -70,10 +70,10 @@ extern "C" int drk_pg_logprob_fwd_noalloc(const void* hidden, const void* W, int
   const bool simt = (in_dtype == DRK_F32) || (engine == DRK_ENGINE_SIMT);
   if (!simt && (H % 8) != 0) return DRK_ERR_UNSUPPORTED;
 
-  // scratch layout: partials [nsplit, T, 2] floats, then target logits [T] floats, each 256-aligned
+  // scratch layout: partials [nsplit, T, 4] floats, then target logits [T] floats, each 256-aligned
   const int ctas = engine == DRK_ENGINE_UMMA_1CTA ? 1 : 2;
   const int nsplit = simt ? simt_nsplit(T, V) : umma_nsplit(T, V, ctas);
-  const size_t part_bytes = align_up(sizeof(float) * 2 * (size_t)nsplit * (size_t)T, 256);
+  const size_t part_bytes = align_up(sizeof(float) * 4 * (size_t)nsplit * (size_t)T, 256);
   const size_t tgt_bytes = align_up(sizeof(float) * (size_t)T, 256);
   if (part_bytes + tgt_bytes > kScratchBytes) return DRK_ERR_WORKSPACE;
 
@@ -92,10 +92,10 @@ extern "C" int drk_pg_logprob_fwd_noalloc(const void* hidden, const void* W, int
   if (cudaMemsetAsync(tgt, 0, tgt_bytes, st) != cudaSuccess) return DRK_ERR_CUDA;
 
   if (simt) {
-    SimtFwdArgs a{hidden, W, in_dtype, ids, T, H, V, logp, lse, part, tgt, nsplit, status};
+    SimtFwdArgs a{hidden, W, in_dtype, ids, T, H, V, logp, lse, part, tgt, nsplit, status, nullptr};
     rc = launch_simt_fwd(a, st);
   } else {
-    UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, part, tgt, nsplit, status, ctas};
+    UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, part, tgt, nsplit, status, ctas, nullptr};
     rc = launch_umma_fwd(a, st);
   }
   if (rc != DRK_OK) g_launches = 0;

@@ -6,8 +6,8 @@
 //                       over the block's vocabulary range, reduced across the 16 lanes that share a
 //                       row with shuffles; the sampled token's logit is written by the one thread
 //                       that owns it.
-//   lse_merge_kernel  : merges the per-range (max, sum-exp) partials into lse and logp (shared with
-//                       the tcgen05 path).
+//   lse_merge_kernel  : merges the per-range (max, sum-exp, sum-exp-times-logit) partials into lse,
+//                       logp and, on request, the token entropy (shared with the tcgen05 path).
 //   lmhead_dl_kernel  : recomputes the tiles of one vocabulary chunk and stores
 //                       dL = c_t (exp(s - lse_t) - onehot) in fp32.
 //   gemm_kernel       : strided fp32 GEMM used for dW = dL^T hidden and dH += dL W.
@@ -66,6 +66,7 @@ __global__ void __launch_bounds__(kThreads)
 lmhead_fwd_kernel(const TIn* __restrict__ hidden, const TIn* __restrict__ W, const int32_t* __restrict__ ids,
                   int64_t T, int H, int V, int tiles_per_split, float* __restrict__ part,
                   float* __restrict__ tgt) {
+  // part holds, per vocabulary range and row, {running max m, sum exp(s-m), sum exp(s-m)*s, unused}
   __shared__ __align__(16) float As[BK][BM + 4];
   __shared__ __align__(16) float Bs[BK][BN + 4];
   const int tid = threadIdx.x, ty = tid / 16, tx = tid % 16;
@@ -74,12 +75,13 @@ lmhead_fwd_kernel(const TIn* __restrict__ hidden, const TIn* __restrict__ W, con
   const int ntiles = (V + BN - 1) / BN;
   const int n_begin = split * tiles_per_split;
   const int n_end = min(ntiles, n_begin + tiles_per_split);
-  float run_m[4], run_l[4];
+  float run_m[4], run_l[4], run_r[4];
   int target[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     run_m[i] = -CUDART_INF_F;
     run_l[i] = 0.f;
+    run_r[i] = 0.f;
     const int64_t r = row0 + ty * 4 + i;
     target[i] = (r < T) ? ids[r] : -1;
   }
@@ -100,15 +102,23 @@ lmhead_fwd_kernel(const TIn* __restrict__ hidden, const TIn* __restrict__ W, con
 #pragma unroll
       for (int o = 8; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
       const float m_new = fmaxf(run_m[i], mx);
-      float s = 0.f;
+      float s = 0.f, sx = 0.f;
       if (m_new > -CUDART_INF_F) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) s += expf(acc[i][j] - m_new);
+        for (int j = 0; j < 4; ++j) {
+          const float e = expf(acc[i][j] - m_new);
+          s += e;
+          sx += e * fmaxf(acc[i][j], -3.0e38f);   // masked columns (-inf) contribute 0, not 0 * inf
+        }
       }
 #pragma unroll
-      for (int o = 8; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      for (int o = 8; o > 0; o >>= 1) {
+        s += __shfl_xor_sync(0xffffffffu, s, o);
+        sx += __shfl_xor_sync(0xffffffffu, sx, o);
+      }
       const float resc = (run_m[i] > -CUDART_INF_F) ? expf(run_m[i] - m_new) : 0.f;
       run_l[i] = run_l[i] * resc + s;
+      run_r[i] = run_r[i] * resc + sx;
       run_m[i] = m_new;
     }
   }
@@ -117,8 +127,7 @@ lmhead_fwd_kernel(const TIn* __restrict__ hidden, const TIn* __restrict__ W, con
     for (int i = 0; i < 4; ++i) {
       const int64_t r = row0 + ty * 4 + i;
       if (r < T) {
-        part[((int64_t)split * T + r) * 2 + 0] = run_m[i];
-        part[((int64_t)split * T + r) * 2 + 1] = run_l[i];
+        reinterpret_cast<float4*>(part)[(int64_t)split * T + r] = make_float4(run_m[i], run_l[i], run_r[i], 0.f);
       }
     }
   }
@@ -126,16 +135,21 @@ lmhead_fwd_kernel(const TIn* __restrict__ hidden, const TIn* __restrict__ W, con
 
 __global__ void lse_merge_kernel(const float* __restrict__ part, const float* __restrict__ tgt,
                                  const int32_t* __restrict__ ids, int64_t T, int V, int nsplit,
-                                 float* __restrict__ logp, float* __restrict__ lse,
+                                 float* __restrict__ logp, float* __restrict__ lse, float* __restrict__ entropy,
                                  uint32_t* __restrict__ status) {
   const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
   if (t >= T) return;
+  const float4* p4 = reinterpret_cast<const float4*>(part);
   float M = -CUDART_INF_F;
-  for (int s = 0; s < nsplit; ++s) M = fmaxf(M, part[((int64_t)s * T + t) * 2]);
-  float L = 0.f;
+  for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p4[(int64_t)s * T + t].x);
+  float L = 0.f, R = 0.f;
   for (int s = 0; s < nsplit; ++s) {
-    const float m = part[((int64_t)s * T + t) * 2], l = part[((int64_t)s * T + t) * 2 + 1];
-    if (m > -CUDART_INF_F) L += l * expf(m - M);
+    const float4 v = p4[(int64_t)s * T + t];
+    if (v.x > -CUDART_INF_F) {
+      const float w = expf(v.x - M);
+      L += v.y * w;
+      R += v.z * w;
+    }
   }
   const float z = M + logf(L);
   const int id = ids[t];
@@ -145,6 +159,7 @@ __global__ void lse_merge_kernel(const float* __restrict__ part, const float* __
   if (!isfinite(z)) bits |= DRK_STATUS_NONFINITE;
   lse[t] = z;
   logp[t] = tg - z;
+  if (entropy != nullptr) entropy[t] = z - R / L;   // H = lse - sum_v p_v s_v
   if (bits) atomicOr(status, bits);
 }
 
@@ -237,8 +252,9 @@ int launch_f32_to_bf16(const float* src, __nv_bfloat16* dst, size_t n, cudaStrea
 }
 
 int launch_lse_merge(const float* part, const float* tgt, const int32_t* ids, int64_t T, int V, int nsplit,
-                     float* logp, float* lse, uint32_t* status, cudaStream_t st) {
-  lse_merge_kernel<<<(unsigned)ceil_div(T, 256), 256, 0, st>>>(part, tgt, ids, T, V, nsplit, logp, lse, status);
+                     float* logp, float* lse, float* entropy, uint32_t* status, cudaStream_t st) {
+  lse_merge_kernel<<<(unsigned)ceil_div(T, 256), 256, 0, st>>>(part, tgt, ids, T, V, nsplit, logp, lse, entropy,
+                                                               status);
   DRK_LAUNCHED();
   return DRK_OK;
 }
@@ -267,7 +283,7 @@ int launch_simt_fwd(const SimtFwdArgs& a, cudaStream_t st) {
                                                                 (const __nv_bfloat16*)a.W, a.ids, a.T, a.H,
                                                                 a.V, per, a.part, a.tgt);
   DRK_LAUNCHED();
-  return launch_lse_merge(a.part, a.tgt, a.ids, a.T, a.V, a.nsplit, a.logp, a.lse, a.status, st);
+  return launch_lse_merge(a.part, a.tgt, a.ids, a.T, a.V, a.nsplit, a.logp, a.lse, a.entropy, a.status, st);
 }
 
 template <typename TIn>

@@ -54,6 +54,7 @@ struct UmmaParams {
   const float* coeff;
   float* part;
   float* tgt;
+  int want_entropy;  // FWD: also carry sum exp(s-m)*s per row
   __nv_bfloat16* dL;
   int vc;
   void* C;
@@ -354,7 +355,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if constexpr (MODE == DH) row_ok = row_ok && orow >= 0;
       }
       // per-unit state
-      float run_m = -CUDART_INF_F, run_l = 0.f;  // FWD: log2-domain running max, sum
+      float run_m = -CUDART_INF_F, run_l = 0.f, run_r = 0.f;  // FWD: log2-domain running max, sum, sum*logit
       int id = -1;
       float c_t = 0.f, z2 = 0.f;
       if constexpr (MODE == FWD) {
@@ -399,9 +400,21 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const float m_new = fmaxf(run_m, cm * kLog2e);
             if (m_new > -CUDART_INF_F) {
               float s = 0.f;
+              const float resc = ex2(run_m - m_new);
+              if (p.want_entropy) {
+                float sx = 0.f;
 #pragma unroll
-              for (int j = 0; j < 32; ++j) s += ex2(fmaf(x[j], kLog2e, -m_new));
-              run_l = run_l * ex2(run_m - m_new) + s;
+                for (int j = 0; j < 32; ++j) {
+                  const float e = ex2(fmaf(x[j], kLog2e, -m_new));
+                  s += e;
+                  sx = fmaf(e, fmaxf(x[j], -3.0e38f), sx);   // masked columns (-inf) contribute 0
+                }
+                run_r = run_r * resc + sx;
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) s += ex2(fmaf(x[j], kLog2e, -m_new));
+              }
+              run_l = run_l * resc + s;
               run_m = m_new;
             }
           } else if constexpr (MODE == DL) {
@@ -452,9 +465,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (!ok) break;
       if constexpr (MODE == FWD) {
         if (row_ok) {
-          float* dst = p.part + ((int64_t)un.j * p.T + row) * 2;
-          dst[0] = run_m * kLn2;  // natural-log units, as the merge kernel expects
-          dst[1] = run_l;
+          // natural-log units for the max, as the merge kernel expects
+          reinterpret_cast<float4*>(p.part)[(int64_t)un.j * p.T + row] = make_float4(run_m * kLn2, run_l, run_r, 0.f);
         }
       }
     }
@@ -618,9 +630,10 @@ int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st) {
   p.group_m = slots / a.nsplit > 0 ? slots / a.nsplit : 1;
   p.rows = a.T; p.cols = a.V; p.v0 = 0; p.T = a.T;
   p.ids = a.ids; p.part = a.part; p.tgt = a.tgt; p.status = a.status;
+  p.want_entropy = a.entropy != nullptr;
   int rc = launch_mode<FWD>(ctas, mh, mw, p, st);
   if (rc != DRK_OK) return rc;
-  return launch_lse_merge(a.part, a.tgt, a.ids, a.T, a.V, a.nsplit, a.logp, a.lse, a.status, st);
+  return launch_lse_merge(a.part, a.tgt, a.ids, a.T, a.V, a.nsplit, a.logp, a.lse, a.entropy, a.status, st);
 }
 
 int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {

@@ -7,7 +7,7 @@ from paper_2602_05885_b200 import binding as B
 
 
 def make_params(lo=None, hi=None, veto=None, norm=0, explicit_scale=1.0, dw_dtype=B.DRK_F32, dh_dtype=B.DRK_F32,
-                dw_accumulate=0, engine=B.DRK_ENGINE_AUTO, v_chunk=0):
+                dw_accumulate=0, engine=B.DRK_ENGINE_AUTO, v_chunk=0, keep_from_caller=0):
     p = B.drk_pg_params_default()
     if lo is not None:
         p.mrs_lo = lo
@@ -22,10 +22,11 @@ def make_params(lo=None, hi=None, veto=None, norm=0, explicit_scale=1.0, dw_dtyp
     p.dw_accumulate = dw_accumulate
     p.engine = engine
     p.v_chunk = v_chunk
+    p.keep_from_caller = keep_from_caller
     return p
 
 
-def run_device(case, p, seg_adv=None, dW_init=None, device="cuda:0"):
+def run_device(case, p, seg_adv=None, dW_init=None, device="cuda:0", keep_in=None):
     dev = torch.device(device)
     hidden = case.hidden.to(dev)
     W = case.W.to(dev)
@@ -42,9 +43,11 @@ def run_device(case, p, seg_adv=None, dW_init=None, device="cuda:0"):
     if dW_init is None:
         bufs.dW.fill_(float("nan"))
     bufs.logp.fill_(float("nan"))
+    if keep_in is not None:
+        bufs.seg_keep.copy_(keep_in.to(dev))
     B.pg_loss_fwd_bwd(hidden, W, ids, rl, mask, cu, adv, p, bufs)
     torch.cuda.synchronize()
-    out = dict(logp=bufs.logp.cpu(), lse=bufs.lse.cpu(), seg_w=bufs.seg_w.cpu(), seg_keep=bufs.seg_keep.cpu(),
+    out = dict(logp=bufs.logp.cpu(), lse=bufs.lse.cpu(), entropy=bufs.entropy.cpu(), seg_w=bufs.seg_w.cpu(), seg_keep=bufs.seg_keep.cpu(),
                loss=bufs.loss.cpu(), counters=bufs.counters.cpu(), dH=bufs.dH.float().cpu(),
                dW=bufs.dW.float().cpu(), status=int(bufs.status.cpu().item()), launches=B.drk_last_launch_count())
     return out

@@ -180,6 +180,9 @@ def check_against_oracle(case: Case, dev: Dict, lo: float, hi: float, veto: floa
         assert err <= tol_logp, f"logp max err {err}"
         err = np.abs(f64(dev["lse"]) - case.lse).max()
         assert err <= tol_logp, f"lse max err {err}"
+        if "entropy" in dev:
+            err = np.abs(f64(dev["entropy"]) - O.token_entropy(case.s)).max()
+            assert err <= tol_logp, f"entropy max err {err}"
     first = oracle_eval(case, lo, hi, veto, norm, explicit_scale, seg_adv=seg_adv, want_grads=False)
     m = first["mrs"]
     keep_dev = dev["seg_keep"].numpy().astype(bool)

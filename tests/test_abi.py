@@ -40,7 +40,7 @@ def test_defaults_are_the_papers_constants():
     assert abs(p.mrs_lo - 0.999) < 1e-7 and abs(p.mrs_hi - 1.001) < 1e-7     # Sec. 5.1 acceptance band
     assert abs(p.veto_ratio - 1e-4) < 1e-10                                     # Sec. 5.1 token veto
     assert p.norm == B.DRK_NORM_KEPT_TOKENS and p.engine == B.DRK_ENGINE_AUTO
-    assert ctypes.sizeof(B.drk_pg_params) == 40
+    assert ctypes.sizeof(B.drk_pg_params) == 44 and p.keep_from_caller == 0
 
 
 def test_workspace_bytes():
@@ -77,7 +77,7 @@ def test_validation_precedes_any_cuda_call():
     assert B.drk_trloo_advantage(z, z, z, 2, 2, 1.0, 9, z, z, z, stream=0, check=False) == B.DRK_ERR_INVALID_ARG
     assert B.drk_trloo_advantage(z, z, z, 2, 65, 1.0, 0, z, z, z, stream=0, check=False) == B.DRK_ERR_UNSUPPORTED
     assert B.drk_trloo_advantage(None, z, z, 2, 2, 1.0, 0, z, z, z, stream=0, check=False) == B.DRK_ERR_INVALID_ARG
-    assert B.drk_pg_logprob_fwd(z, z, B.DRK_BF16, z, 8, 0, 16, 0, z, z, z, 1 << 20, z, stream=0,
+    assert B.drk_pg_logprob_fwd(z, z, B.DRK_BF16, z, 8, 0, 16, 0, z, z, None, z, 1 << 20, z, stream=0,
                                 check=False) == B.DRK_ERR_INVALID_ARG
     assert B.drk_last_launch_count() == 0
 

@@ -52,12 +52,12 @@ def test_empty_inputs():
     e = torch.empty(0, device=d)
     cu = torch.zeros(3, dtype=torch.int32, device=d)
     B.drk_pg_loss_fwd_bwd(e, W, B.DRK_BF16, e, e, e, cu, torch.ones(2, device=d), 0, H, V, 2, p, bufs.loss, bufs.logp,
-                          bufs.lse, bufs.seg_w, bufs.seg_keep, bufs.counters, bufs.dH, bufs.dW, bufs.workspace,
+                          bufs.lse, None, bufs.seg_w, bufs.seg_keep, bufs.counters, bufs.dH, bufs.dW, bufs.workspace,
                           bufs.workspace_bytes, bufs.status)
     torch.cuda.synchronize()
     assert float(bufs.loss.item()) == 0.0 and (bufs.dW == 0).all() and (bufs.seg_keep == 0).all()
     assert (bufs.seg_w == 1).all()
-    assert B.drk_pg_logprob_fwd(e, W, B.DRK_BF16, e, 0, H, V, 0, e, e, bufs.workspace, bufs.workspace_bytes,
+    assert B.drk_pg_logprob_fwd(e, W, B.DRK_BF16, e, 0, H, V, 0, e, e, None, bufs.workspace, bufs.workspace_bytes,
                                 bufs.status) == B.DRK_OK
 
 
@@ -92,7 +92,7 @@ def test_host_detected_errors_return_codes():
     nb = B.drk_pg_workspace_bytes(T, H, V, 0, B.DRK_BF16, None, 0)
     ws = torch.empty(nb, dtype=torch.uint8, device=d)
     call = lambda **kw: B.drk_pg_logprob_fwd(kw.get("hidden", hidden), W, kw.get("dt", B.DRK_BF16), ids,
-                                             kw.get("T", T), kw.get("H", H), V, 0, logp, lse, ws,
+                                             kw.get("T", T), kw.get("H", H), V, 0, logp, lse, None, ws,
                                              kw.get("nb", nb), st, check=False)
     assert call() == B.DRK_OK
     assert call(nb=nb - 512) == B.DRK_ERR_WORKSPACE

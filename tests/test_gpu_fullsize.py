@@ -43,7 +43,7 @@ def _run(wl, p, seg_adv):
     dev = wl.hidden.device
     bufs = B.PgLossBuffers(wl.T, wl.H, wl.V, wl.S, B.DRK_BF16, p, dev)
     B.drk_pg_loss_fwd_bwd(wl.hidden, wl.W, B.DRK_BF16, wl.ids, wl.rollout_logp, wl.loss_mask, wl.cu, seg_adv,
-                          wl.T, wl.H, wl.V, wl.S, p, bufs.loss, bufs.logp, bufs.lse, bufs.seg_w, bufs.seg_keep,
+                          wl.T, wl.H, wl.V, wl.S, p, bufs.loss, bufs.logp, bufs.lse, bufs.entropy, bufs.seg_w, bufs.seg_keep,
                           bufs.counters, bufs.dH, bufs.dW, bufs.workspace, bufs.workspace_bytes, bufs.status)
     torch.cuda.synchronize()
     assert int(bufs.status.item()) == 0

@@ -118,3 +118,20 @@ def test_end_to_end_with_device_advantages():
     lo, hi = Hh.wide_band(case)
     dev = run_device(case, make_params(lo, hi, PAPER[2]), seg_adv=seg_adv_dev)
     Hh.check_against_oracle(case, dev, lo, hi, PAPER[2])
+
+
+def test_keep_flags_from_the_caller():
+    # the caller decides retention (e.g. samples split over micro-batches): seg_keep is an input
+    case = get_case("medium")
+    g = torch.Generator().manual_seed(3)
+    keep_in = (torch.rand(case.S, generator=g) < 0.6).to(torch.uint8)
+    dev = run_device(case, make_params(*PAPER, keep_from_caller=1), keep_in=keep_in)
+    assert torch.equal(dev["seg_keep"], keep_in)
+    ref = Hh.oracle_eval(case, *PAPER, keep_override=keep_in.numpy())
+    assert dev["counters"][0] == ref["kept_tokens"] and dev["counters"][2] == ref["kept_segs"] == int(keep_in.sum())
+    denom = max(abs(ref["loss"]), 1e-3 * float(np.sum(np.abs(ref["coeff"] * case.logp))))
+    assert abs(float(dev["loss"]) - ref["loss"]) / denom <= Hh.TOL_LOSS_REL
+    assert Hh.rel_fro(Hh.f64(dev["dH"]), ref["dH"]) <= Hh.TOL_GRAD_FRO
+    assert Hh.rel_fro(Hh.f64(dev["dW"]), ref["dW"]) <= Hh.TOL_GRAD_FRO
+    # seg_w is still this micro-batch's geometric-mean ratio
+    assert np.abs(Hh.f64(dev["seg_w"]) - ref["mrs"].w).max() <= 2 * Hh.TOL_LOGP_BF16
