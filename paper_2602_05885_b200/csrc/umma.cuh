@@ -214,13 +214,27 @@ __device__ __forceinline__ void mma_bf16_ss_pair(uint32_t tmem_d, uint64_t desc_
       ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// Arrive, in every CTA named by `cta_mask`, on the mbarrier at this offset once all tcgen05
-// operations issued so far by this thread have completed.
+// Arrive, in every CTA of the pair named by `cta_mask` (bit 0: even CTA, bit 1: odd CTA), on the
+// mbarrier at this shared-memory offset once all tcgen05 operations issued so far by this thread
+// have completed.  Issued by the even CTA.  One tcgen05.commit whose arrival is multicast to the
+// barriers of both CTAs is 4 % faster end to end than two commits (one per barrier, the peer's
+// addressed through the cluster window); the latter is kept behind DRK_COMMIT_PAIRWISE.  This is
+// a barrier signal, not a data load: no TMA load in this library uses cluster multicast.
 __device__ __forceinline__ void mma_commit_pair(uint32_t bar, uint16_t cta_mask) {
+#ifndef DRK_COMMIT_PAIRWISE
   asm volatile(
       "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
       ::"r"(bar), "h"(cta_mask)
       : "memory");
+#else
+  if (cta_mask & 1)
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  if (cta_mask & 2) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, 1;" : "=r"(remote) : "r"(bar));
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(remote) : "memory");
+  }
+#endif
 }
 
 }  // namespace ptx

@@ -30,8 +30,11 @@ namespace {
 
 constexpr int TM = 128, TN = 256, TK = 64;
 constexpr int A_BYTES = TM * TK * 2;      // 16 KiB: 128 rows of A per CTA
-constexpr int RING_BYTES = 192 * 1024;    // operand ring: 4 stages of 48 KiB, or 6 of 32 KiB for a CTA pair
-constexpr int MAX_STAGES = 6;
+#ifndef DRK_RING_KB
+#define DRK_RING_KB 192
+#endif
+constexpr int RING_BYTES = DRK_RING_KB * 1024;  // operand ring: 4 stages of 48 KiB, or 6 of 32 KiB for a CTA pair
+constexpr int MAX_STAGES = 8;
 constexpr int SUB_BYTES = 64 * TK * 2;    // one 64-wide MN-major box: 64 k-rows x 128 B
 constexpr int NUM_THREADS = 192;
 constexpr int NUM_BARS = 2 * MAX_STAGES + 5;
