@@ -11,7 +11,7 @@
 //   DH  : dH (+)= dL W[chunk]               (A K-major, B MN-major)
 //
 // Tile 128 x 256 x 64, one CTA per SM, 192 threads:
-//   warp 0    : TMA producer (one lane): 128B-swizzled operand tiles into a 4-stage ring
+//   warp 0    : TMA producer (one lane): 128B-swizzled operand tiles into a ring of stages
 //   warp 1    : tensor-memory allocation; one lane issues tcgen05.mma (4 per stage, K = 16 each)
 //               into one of two 256-column fp32 accumulators and commits to mbarriers
 //   warps 2-5 : epilogue; warp w reads tensor-memory lanes 32*(w%4)..+31, one accumulator row per
@@ -30,6 +30,13 @@ namespace {
 
 constexpr int TM = 128, TN = 256, TK = 64;
 constexpr int A_BYTES = TM * TK * 2;      // 16 KiB: 128 rows of A per CTA
+// 64-deep k-blocks per pipeline stage of a CTA pair.  Two (three 64 KiB stages, eight MMAs per
+// tcgen05.commit) measured 4 % faster end to end than one (six 32 KiB stages, four MMAs per commit).
+// The backward's row padding (256 rows) covers at most four k-blocks per stage.
+#ifndef DRK_STAGE_SUBS
+#define DRK_STAGE_SUBS 2
+#endif
+static_assert(DRK_STAGE_SUBS == 1 || DRK_STAGE_SUBS == 2 || DRK_STAGE_SUBS == 4, "stage depth must divide the 256-row padding");
 #ifndef DRK_RING_KB
 #define DRK_RING_KB 192
 #endif
@@ -183,8 +190,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   constexpr uint32_t IDESC = ptx::make_idesc_bf16(TM * CTAS, TN, A_MN ? 1 : 0, B_MN ? 1 : 0);
   constexpr int BN_CTA = TN / CTAS;                 // rows of B this CTA loads
   constexpr int B_BYTES_CTA = BN_CTA * TK * 2;
-  constexpr int STAGE = A_BYTES + B_BYTES_CTA;      // bytes per stage in this CTA
-  constexpr int NSTAGE = RING_BYTES / STAGE;        // 4 (one CTA) or 6 (pair)
+  constexpr int SUBS = (CTAS == 2) ? DRK_STAGE_SUBS : 1;  // 64-deep k-blocks per pipeline stage
+  constexpr int SUB = A_BYTES + B_BYTES_CTA;        // bytes of one k-block (A rows + B rows of this CTA)
+  constexpr int STAGE = SUBS * SUB;                 // bytes per stage in this CTA
+  constexpr int NSTAGE = RING_BYTES / STAGE;
   constexpr uint32_t TX_BYTES = STAGE * CTAS;       // both CTAs' loads are credited to one barrier
 
   extern __shared__ uint8_t smem_raw[];
@@ -264,25 +273,30 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int a_row = (un.m * CTAS + cta_rank) * TM;   // first A row (M index) of this CTA
         for (int n = un.n_begin; n < un.n_end && ok; ++n) {
           const int b_row = n * TN + cta_rank * BN_CTA;     // first B row (N index) of this CTA
-          for (int kb = 0; kb < k_blocks; ++kb) {
+          for (int kb0 = 0; kb0 < k_blocks; kb0 += SUBS) {
             const int s = it % NSTAGE;
             const uint32_t ph = (it / NSTAGE) & 1u;
             if (!ptx::mbar_wait(empty_bar(s), ph ^ 1u, abort, WAIT_LIMIT_NS)) { ok = false; break; }
             if (leader) ptx::mbar_arrive_expect_tx(full_bar(s), TX_BYTES);
-            const uint32_t sa = smem_base + s * STAGE, sb = sa + A_BYTES;
-            if constexpr (MODE == FWD || MODE == DL) {
-              load(sa, &tmA, full_bar(s), kb * TK, a_row);
-              load(sb, &tmB, full_bar(s), kb * TK, p.v0 + b_row);
-            } else if constexpr (MODE == DW) {
 #pragma unroll
-              for (int j = 0; j < TM / 64; ++j) load(sa + j * SUB_BYTES, &tmA, full_bar(s), a_row + 64 * j, kb * TK);
+            for (int sub = 0; sub < SUBS; ++sub) {
+              // a k-block past the end of K lies outside the tensor and is filled with zeros
+              const int kb = kb0 + sub;
+              const uint32_t sa = smem_base + s * STAGE + sub * SUB, sb = sa + A_BYTES;
+              if constexpr (MODE == FWD || MODE == DL) {
+                load(sa, &tmA, full_bar(s), kb * TK, a_row);
+                load(sb, &tmB, full_bar(s), kb * TK, p.v0 + b_row);
+              } else if constexpr (MODE == DW) {
 #pragma unroll
-              for (int j = 0; j < BN_CTA / 64; ++j) load(sb + j * SUB_BYTES, &tmB, full_bar(s), b_row + 64 * j, kb * TK);
-            } else {  // DH
-              load(sa, &tmA, full_bar(s), kb * TK, a_row);
+                for (int j = 0; j < TM / 64; ++j) load(sa + j * SUB_BYTES, &tmA, full_bar(s), a_row + 64 * j, kb * TK);
 #pragma unroll
-              for (int j = 0; j < BN_CTA / 64; ++j)
-                load(sb + j * SUB_BYTES, &tmB, full_bar(s), b_row + 64 * j, p.v0 + kb * TK);
+                for (int j = 0; j < BN_CTA / 64; ++j) load(sb + j * SUB_BYTES, &tmB, full_bar(s), b_row + 64 * j, kb * TK);
+              } else {  // DH
+                load(sa, &tmA, full_bar(s), kb * TK, a_row);
+#pragma unroll
+                for (int j = 0; j < BN_CTA / 64; ++j)
+                  load(sb + j * SUB_BYTES, &tmB, full_bar(s), b_row + 64 * j, p.v0 + kb * TK);
+              }
             }
             ++it;
           }
@@ -312,22 +326,26 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           if (!ptx::mbar_wait(tempty_bar(acc), aph ^ 1u, abort, WAIT_LIMIT_NS)) { ok = false; break; }
           ptx::tc_fence_after();
           const uint32_t d_tmem = tmem_base + acc * TN;
-          for (int kb = 0; kb < k_blocks; ++kb) {
+          for (int kb0 = 0; kb0 < k_blocks; kb0 += SUBS) {
             const int s = it % NSTAGE;
             const uint32_t ph = (it / NSTAGE) & 1u;
             if (!ptx::mbar_wait(full_bar(s), ph, abort, WAIT_LIMIT_NS)) { ok = false; break; }
             ptx::tc_fence_after();
-            const uint32_t sa = smem_base + s * STAGE, sb = sa + A_BYTES;
 #pragma unroll
-            for (int k = 0; k < TK / 16; ++k) {
-              // K-major: 16 elements = 32 B further along the swizzled 128 B row.
-              // MN-major: 16 k-rows of 128 B = two 8-row swizzle atoms further.
-              const uint64_t da = A_MN ? ptx::make_smem_desc(sa + k * 2048, SUB_BYTES, 1024)
-                                       : ptx::make_smem_desc(sa + k * 32, 16, 1024);
-              const uint64_t db = B_MN ? ptx::make_smem_desc(sb + k * 2048, SUB_BYTES, 1024)
-                                       : ptx::make_smem_desc(sb + k * 32, 16, 1024);
-              if constexpr (CTAS == 2) ptx::mma_bf16_ss_pair(d_tmem, da, db, IDESC, (kb | k) != 0 ? 1u : 0u);
-              else ptx::mma_bf16_ss(d_tmem, da, db, IDESC, (kb | k) != 0 ? 1u : 0u);
+            for (int sub = 0; sub < SUBS; ++sub) {
+              const uint32_t sa = smem_base + s * STAGE + sub * SUB, sb = sa + A_BYTES;
+#pragma unroll
+              for (int k = 0; k < TK / 16; ++k) {
+                // K-major: 16 elements = 32 B further along the swizzled 128 B row.
+                // MN-major: 16 k-rows of 128 B = two 8-row swizzle atoms further.
+                const uint64_t da = A_MN ? ptx::make_smem_desc(sa + k * 2048, SUB_BYTES, 1024)
+                                         : ptx::make_smem_desc(sa + k * 32, 16, 1024);
+                const uint64_t db = B_MN ? ptx::make_smem_desc(sb + k * 2048, SUB_BYTES, 1024)
+                                         : ptx::make_smem_desc(sb + k * 32, 16, 1024);
+                const uint32_t accum = (kb0 | sub | k) != 0 ? 1u : 0u;
+                if constexpr (CTAS == 2) ptx::mma_bf16_ss_pair(d_tmem, da, db, IDESC, accum);
+                else ptx::mma_bf16_ss(d_tmem, da, db, IDESC, accum);
+              }
             }
             commit(empty_bar(s));  // frees the stage (in both CTAs) once these MMAs have read it
             ++it;
