@@ -340,6 +340,12 @@ def main():
     flops = (2.0 * T + 6.0 * Tc) * H * V
     peaks = measured_peaks()
     achieved = flops / (fused_ms * 1e-3) / 1e12
+    # DRAM bytes of one fused call from the committed one-pass ncu capture of exactly this configuration
+    # (profiles/umma_gemm_kernel_pairs_T32768_onepass.md); unknown for any other configuration.
+    traffic = None
+    if (args.workload, T, args.mrs, args.dw_dtype, args.dh_dtype, args.v_chunk, args.engine) == \
+            ("qwen3-14b", 32768, "wide", "f32", "bf16", 0, "auto"):
+        traffic = 260.87e9
     # the same call with rejection switched off: every loss-masked token goes through the backward
     p_off = B.drk_pg_params_default()
     ctypes_copy = [f[0] for f in p._fields_]
@@ -405,7 +411,7 @@ def main():
                        "l2": "inputs exceed L2 (W alone is %.2f GB); no flush" % (V * H * 2 / 1e9),
                        "parallelism": f"dp{world}: one micro-batch per rank, no collective on the loss path"},
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s",
-                         "frac": achieved / peaks["tflops"], "traffic": None,
+                         "frac": achieved / peaks["tflops"], "traffic": traffic,
                          "kernel": "umma_gemm_kernel (all four instantiations inside one drk_pg_loss_fwd_bwd call)",
                          "flops_per_call": flops, "call_ms": fused_ms, "gemm_launches_per_call": n_gemm_launches,
                          "flops_rule": "(2 T + 6 Tc) H V: forward over all T rows, backward over the Tc rows with "
