@@ -24,3 +24,11 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_library():
+    """Build libdrk.so once per session if it is missing or older than its sources (needs nvcc only)."""
+    from paper_2602_05885_b200 import build
+    build.build_library()
+    yield

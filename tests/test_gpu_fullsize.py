@@ -129,12 +129,13 @@ def test_full_size_structured_rows():
     assert err <= Hh.TOL_GRAD_FRO, f"dW rel Frobenius err {err}"
 
 
-@pytest.mark.parametrize("shape", [None, (4096, 32768, 4096), (65536, 151936, 5120)],
-                         ids=["bench-14b", "sweep-smallest", "sweep-largest"])
+@pytest.mark.parametrize("shape", ["qwen3-14b", "qwen3-8b", "ragged", (4096, 32768, 4096), (65536, 151936, 5120)],
+                         ids=["bench-14b", "full-8b", "full-ragged", "sweep-smallest", "sweep-largest"])
 def test_full_size_bench_inputs_sampled_rows(shape):
-    """The benchmark's own 14B-shaped micro-batch, and the smallest and largest points of the roofline sweep."""
+    """The benchmark's own 14B-shaped micro-batch, the 8B-shaped and the ragged multi-turn micro-batches at
+    full size, and the smallest and largest points of the roofline sweep."""
     dev = torch.device("cuda:0")
-    wl = workload.build("qwen3-14b", dev, seed=2000) if shape is None else \
+    wl = workload.build(shape, dev, seed=2000) if isinstance(shape, str) else \
         workload.build("sweep", dev, seed=4000, sweep_shape=shape)
     T, H, V, S = wl.T, wl.H, wl.V, wl.S
     # MRS off and an explicit scale: every coefficient is then known without the other rows' log-probs
@@ -159,6 +160,7 @@ def test_full_size_bench_inputs_sampled_rows(shape):
     logp, lse = O.token_logprob(s, ids)
     assert np.abs(Hh.f64(bufs.logp)[sample] - logp).max() <= Hh.TOL_LOGP_BF16
     assert np.abs(Hh.f64(bufs.lse)[sample] - lse).max() <= Hh.TOL_LOGP_BF16
+    assert np.abs(Hh.f64(bufs.entropy)[sample] - O.token_entropy(s)).max() <= Hh.TOL_LOGP_BF16
     dH_s, _ = O.gradients(hid, W64, s, lse, ids, lr.coeff[sample])
     assert Hh.rel_fro(Hh.f64(bufs.dH[st.to(dev)]), dH_s) <= Hh.TOL_GRAD_FRO
     # every row of softmax - onehot sums to zero, hence so do the columns of dW over the vocabulary
