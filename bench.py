@@ -216,6 +216,8 @@ def main():
     ap.add_argument("--dw-dtype", default="f32", choices=["f32", "bf16"])
     ap.add_argument("--dh-dtype", default="bf16", choices=["f32", "bf16"])
     ap.add_argument("--v-chunk", type=int, default=0)
+    ap.add_argument("--forward-rows", default="all", choices=["all", "usable"],
+                    help="usable: the forward skips rows that are not loss-masked tokens of a segment")
     ap.add_argument("--engine", default="auto", choices=["auto", "1cta"],
                     help="auto: tcgen05 kernels on CTA pairs; 1cta: one CTA per tile")
     ap.add_argument("--mrs", default="wide", choices=["wide", "paper", "off"])
@@ -262,6 +264,7 @@ def main():
     p.dh_dtype = B.DRK_BF16 if args.dh_dtype == "bf16" else B.DRK_F32
     p.v_chunk = args.v_chunk
     p.engine = B.DRK_ENGINE_UMMA_1CTA if args.engine == "1cta" else B.DRK_ENGINE_AUTO
+    p.forward_rows = 1 if args.forward_rows == "usable" else 0
     bufs = B.PgLossBuffers(T, H, V, S, code, p, dev)
     R, Tmax = wl.reward.shape
     ret = torch.empty_like(wl.reward)
@@ -337,14 +340,15 @@ def main():
     # merge + 3 MRS + 4 compaction kernels are not GEMM launches (the FFMA path has no compaction)
     n_gemm_launches = B.drk_last_launch_count() - (8 if code == B.DRK_BF16 else 4)
     Tc = backward_rows() if code == B.DRK_BF16 else T
-    flops = (2.0 * T + 6.0 * Tc) * H * V
+    Tf = int(bufs.counters[1].item()) if (p.forward_rows == 1 and code == B.DRK_BF16) else T   # rows the forward ran on
+    flops = (2.0 * Tf + 6.0 * Tc) * H * V
     peaks = measured_peaks()
     achieved = flops / (fused_ms * 1e-3) / 1e12
     # DRAM bytes of one fused call from the committed one-pass ncu capture of exactly this configuration
     # (profiles/umma_gemm_kernel_pairs_T32768_onepass.md); unknown for any other configuration.
     traffic = None
-    if (args.workload, T, args.mrs, args.dw_dtype, args.dh_dtype, args.v_chunk, args.engine) == \
-            ("qwen3-14b", 32768, "wide", "f32", "bf16", 0, "auto"):
+    if (args.workload, T, args.mrs, args.dw_dtype, args.dh_dtype, args.v_chunk, args.engine, args.forward_rows) == \
+            ("qwen3-14b", 32768, "wide", "f32", "bf16", 0, "auto", "all"):
         traffic = 260.87e9
     # the same call with rejection switched off: every loss-masked token goes through the backward
     p_off = B.drk_pg_params_default()
@@ -354,7 +358,7 @@ def main():
     p_off.mrs_lo, p_off.mrs_hi, p_off.veto_ratio = 0.0, float("inf"), 0.0
     off_ms = time_fused(p_off, min(args.steps, 5))
     Tc_off = backward_rows() if code == B.DRK_BF16 else T
-    off_tflops = (2.0 * T + 6.0 * Tc_off) * H * V / (off_ms * 1e-3) / 1e12
+    off_tflops = (2.0 * Tf + 6.0 * Tc_off) * H * V / (off_ms * 1e-3) / 1e12
     time_fused(p, 1)   # leave the outputs of the configured run in the buffers
 
     # ---------------------------------------------------------------- end to end with host buffers
@@ -407,7 +411,7 @@ def main():
             "config": {"workload": f"{wl.name}-shaped packed micro-batch", "T": T, "H": H, "V": V, "segments": S,
                        "rollout_batch": f"{R} rollouts x {Tmax} turns", "mrs": args.mrs,
                        "dW": args.dw_dtype, "dH": args.dh_dtype, "v_chunk": args.v_chunk or "default",
-                       "engine": args.engine,
+                       "engine": args.engine, "forward_rows": args.forward_rows,
                        "l2": "inputs exceed L2 (W alone is %.2f GB); no flush" % (V * H * 2 / 1e9),
                        "parallelism": f"dp{world}: one micro-batch per rank, no collective on the loss path"},
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s",
@@ -416,7 +420,7 @@ def main():
                          "flops_per_call": flops, "call_ms": fused_ms, "gemm_launches_per_call": n_gemm_launches,
                          "flops_rule": "(2 T + 6 Tc) H V: forward over all T rows, backward over the Tc rows with "
                                        "a non-zero coefficient (rows of rejected or masked tokens are skipped)",
-                         "rows_in_backward": Tc,
+                         "rows_in_backward": Tc, "rows_in_forward": Tf,
                          "no_rejection": {"call_ms": off_ms, "rows_in_backward": Tc_off, "tflops": off_tflops,
                                           "frac": off_tflops / peaks["tflops"],
                                           "tokens_per_s": T / (off_ms * 1e-3)},

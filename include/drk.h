@@ -132,6 +132,10 @@ typedef struct {
                             split over several micro-batches, judged on log-probs from
                             drk_pg_logprob_fwd of all its pieces); seg_w and the counters are still
                             computed from this micro-batch's tokens                                   */
+  int32_t forward_rows;  /* 0: log-probs of all T rows.  1: only of the rows the loss can use (loss-masked
+                            tokens inside segments); logp, lse, entropy of every other row read 0.  Saves the
+                            forward's work on prompt / feedback / padding tokens; tensor-core path only
+                            (ignored by the FFMA path)                                                  */
 } drk_pg_params;
 
 void drk_pg_params_default(drk_pg_params* p); /* host pointer */

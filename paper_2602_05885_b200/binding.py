@@ -52,6 +52,7 @@ class drk_pg_params(ctypes.Structure):
         ("engine", ctypes.c_int32),
         ("v_chunk", ctypes.c_int32),
         ("keep_from_caller", ctypes.c_int32),
+        ("forward_rows", ctypes.c_int32),
     ]
 
 

@@ -130,6 +130,7 @@ bool params_ok(const drk_pg_params& p) {
   if (!engine_ok(p.engine)) return false;
   if (p.v_chunk < 0) return false;
   if (p.keep_from_caller != 0 && p.keep_from_caller != 1) return false;
+  if (p.forward_rows != 0 && p.forward_rows != 1) return false;
   if (std::isnan(p.mrs_lo) || std::isnan(p.mrs_hi) || std::isnan(p.veto_ratio)) return false;
   if (p.norm == DRK_NORM_EXPLICIT && !std::isfinite(p.explicit_scale)) return false;
   return true;
@@ -137,12 +138,14 @@ bool params_ok(const drk_pg_params& p) {
 
 int run_fwd(const void* hidden, const void* W, int in_dtype, const int32_t* ids, int64_t T, int H, int V,
             bool simt, int engine, const FwdWs& w, float* logp, float* lse, float* entropy, uint32_t* status,
-            cudaStream_t st) {
+            cudaStream_t st, const __nv_bfloat16* hidden_c = nullptr, const int32_t* rowmap = nullptr,
+            const int32_t* n_rows = nullptr) {
   if (simt) {
     SimtFwdArgs a{hidden, W, in_dtype, ids, T, H, V, logp, lse, w.part, w.tgt, w.nsplit, status, entropy};
     return launch_simt_fwd(a, st);
   }
-  UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, w.part, w.tgt, w.nsplit, status, umma_ctas(engine), entropy};
+  UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, w.part, w.tgt, w.nsplit, status, umma_ctas(engine), entropy,
+                hidden_c, rowmap, n_rows};
   return launch_umma_fwd(a, st);
 }
 
@@ -166,6 +169,7 @@ void drk_pg_params_default(drk_pg_params* p) {
   p->engine = DRK_ENGINE_AUTO;
   p->v_chunk = 0;
   p->keep_from_caller = 0;
+  p->forward_rows = 0;
 }
 
 size_t drk_pg_workspace_bytes(int64_t T, int32_t H, int32_t V, int32_t S, int32_t in_dtype,
@@ -252,7 +256,22 @@ int drk_pg_loss_fwd_bwd(const void* hidden, const void* W, int32_t in_dtype, con
 
   auto fail = [&](int code) { g_launches = 0; return code; };
 
-  if (T > 0) {
+  if (T > 0 && p.forward_rows == 1 && !simt) {
+    // forward over the rows the loss can use: loss-masked tokens inside segments; the rest read 0
+    rc = launch_need_rows(loss_mask, cu_seqlens, T, S, bw.coeff, st);
+    if (rc != DRK_OK) return fail(rc);
+    CompactArgs ca{bw.coeff, static_cast<const __nv_bfloat16*>(hidden), T, H, bw.blk_cnt, bw.blk_off, bw.n_rows,
+                   bw.rowmap, bw.hidden_c};
+    rc = launch_compact(ca, st);
+    if (rc != DRK_OK) return fail(rc);
+    if (cudaMemsetAsync(logp, 0, sizeof(float) * (size_t)T, st) != cudaSuccess ||
+        cudaMemsetAsync(lse, 0, sizeof(float) * (size_t)T, st) != cudaSuccess ||
+        (entropy && cudaMemsetAsync(entropy, 0, sizeof(float) * (size_t)T, st) != cudaSuccess))
+      return fail(DRK_ERR_CUDA);
+    rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, p.engine, fw, logp, lse, entropy, status, st, bw.hidden_c,
+                 bw.rowmap, bw.n_rows);
+    if (rc != DRK_OK) return fail(rc);
+  } else if (T > 0) {
     rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, p.engine, fw, logp, lse, entropy, status, st);
     if (rc != DRK_OK) return fail(rc);
   }

@@ -55,7 +55,8 @@ struct SimtFwdArgs {
 int simt_nsplit(int64_t T, int V);
 int launch_simt_fwd(const SimtFwdArgs& a, cudaStream_t st);
 int launch_lse_merge(const float* part, const float* tgt, const int32_t* ids, int64_t T, int V, int nsplit,
-                     float* logp, float* lse, float* entropy, uint32_t* status, cudaStream_t st);
+                     float* logp, float* lse, float* entropy, uint32_t* status, const int32_t* rowmap,
+                     const int32_t* n_rows, cudaStream_t st);
 struct SimtBwdArgs {
   const void* hidden; const void* W; int in_dtype; const int32_t* ids; int64_t T; int H; int V;
   const float* lse; const float* coeff; float* dL /*[T*vc] fp32 workspace*/; int vc;
@@ -70,6 +71,8 @@ struct UmmaFwdArgs {
   float* logp; float* lse; float* part /*[nsplit*T*4]*/; float* tgt; int nsplit; uint32_t* status;
   int ctas /*1: one CTA per tile; 2: CTA pairs*/;
   float* entropy /*[T] or null*/;
+  // optional: evaluate only the rows listed in rowmap (gathered into hidden_c); others are left untouched
+  const __nv_bfloat16* hidden_c; const int32_t* rowmap; const int32_t* n_rows;
 };
 int umma_nsplit(int64_t T, int V, int ctas);
 int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st);
@@ -91,6 +94,8 @@ struct CompactArgs {
 int64_t compact_map_len(int64_t T);
 int compact_blocks(int64_t T);
 int launch_compact(const CompactArgs& a, cudaStream_t st);
+// need[t] = 1 for loss-masked tokens inside a segment, else 0 (the rows whose log-prob the loss can use)
+int launch_need_rows(const uint8_t* loss_mask, const int32_t* cu, int64_t T, int S, float* need, cudaStream_t st);
 
 // Small utility kernels.
 int launch_f32_to_bf16(const float* src, __nv_bfloat16* dst, size_t n, cudaStream_t st);

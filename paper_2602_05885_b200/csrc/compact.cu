@@ -74,6 +74,23 @@ __global__ void __launch_bounds__(256) gather_kernel(const __nv_bfloat16* __rest
   }
 }
 
+__global__ void __launch_bounds__(256) need_rows_kernel(const uint8_t* __restrict__ mask, const int32_t* __restrict__ cu,
+                                                        int64_t T, float* __restrict__ need) {
+  const int g = blockIdx.x;
+  const int64_t a = cu[g], b = cu[g + 1];
+  if (a < 0 || b < a || b > T) return;
+  for (int64_t t = a + threadIdx.x; t < b; t += blockDim.x) need[t] = mask[t] ? 1.f : 0.f;
+}
+
+int launch_need_rows(const uint8_t* loss_mask, const int32_t* cu, int64_t T, int S, float* need, cudaStream_t st) {
+  if (T == 0) return DRK_OK;
+  DRK_CUDA_CHECK(cudaMemsetAsync(need, 0, sizeof(float) * (size_t)T, st));
+  if (S == 0) return DRK_OK;
+  need_rows_kernel<<<S, 256, 0, st>>>(loss_mask, cu, T, need);
+  DRK_LAUNCHED();
+  return DRK_OK;
+}
+
 int64_t compact_map_len(int64_t T) { return (T + 255) / 256 * 256 + 256; }
 int compact_blocks(int64_t T) { return (int)((compact_map_len(T) + kBlk - 1) / kBlk); }
 

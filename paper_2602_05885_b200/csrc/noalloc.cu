@@ -95,7 +95,7 @@ extern "C" int drk_pg_logprob_fwd_noalloc(const void* hidden, const void* W, int
     SimtFwdArgs a{hidden, W, in_dtype, ids, T, H, V, logp, lse, part, tgt, nsplit, status, nullptr};
     rc = launch_simt_fwd(a, st);
   } else {
-    UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, part, tgt, nsplit, status, ctas, nullptr};
+    UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, part, tgt, nsplit, status, ctas, nullptr, nullptr, nullptr, nullptr};
     rc = launch_umma_fwd(a, st);
   }
   if (rc != DRK_OK) g_launches = 0;

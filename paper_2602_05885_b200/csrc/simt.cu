@@ -136,15 +136,22 @@ lmhead_fwd_kernel(const TIn* __restrict__ hidden, const TIn* __restrict__ W, con
 __global__ void lse_merge_kernel(const float* __restrict__ part, const float* __restrict__ tgt,
                                  const int32_t* __restrict__ ids, int64_t T, int V, int nsplit,
                                  float* __restrict__ logp, float* __restrict__ lse, float* __restrict__ entropy,
-                                 uint32_t* __restrict__ status) {
-  const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-  if (t >= T) return;
+                                 uint32_t* __restrict__ status, const int32_t* __restrict__ rowmap,
+                                 const int32_t* __restrict__ n_rows) {
+  // r: row of the partials; t: the token it belongs to (they differ when the forward ran on gathered rows)
+  const int64_t r = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (r >= T) return;
+  int64_t t = r;
+  if (rowmap != nullptr) {
+    if (r >= n_rows[0]) return;
+    t = rowmap[r];
+  }
   const float4* p4 = reinterpret_cast<const float4*>(part);
   float M = -CUDART_INF_F;
-  for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p4[(int64_t)s * T + t].x);
+  for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p4[(int64_t)s * T + r].x);
   float L = 0.f, R = 0.f;
   for (int s = 0; s < nsplit; ++s) {
-    const float4 v = p4[(int64_t)s * T + t];
+    const float4 v = p4[(int64_t)s * T + r];
     if (v.x > -CUDART_INF_F) {
       const float w = expf(v.x - M);
       L += v.y * w;
@@ -155,7 +162,7 @@ __global__ void lse_merge_kernel(const float* __restrict__ part, const float* __
   const int id = ids[t];
   uint32_t bits = 0;
   float tg = 0.f;
-  if (id >= 0 && id < V) tg = tgt[t]; else bits |= DRK_STATUS_BAD_ID;
+  if (id >= 0 && id < V) tg = tgt[r]; else bits |= DRK_STATUS_BAD_ID;
   if (!isfinite(z)) bits |= DRK_STATUS_NONFINITE;
   lse[t] = z;
   logp[t] = tg - z;
@@ -252,9 +259,10 @@ int launch_f32_to_bf16(const float* src, __nv_bfloat16* dst, size_t n, cudaStrea
 }
 
 int launch_lse_merge(const float* part, const float* tgt, const int32_t* ids, int64_t T, int V, int nsplit,
-                     float* logp, float* lse, float* entropy, uint32_t* status, cudaStream_t st) {
+                     float* logp, float* lse, float* entropy, uint32_t* status, const int32_t* rowmap,
+                     const int32_t* n_rows, cudaStream_t st) {
   lse_merge_kernel<<<(unsigned)ceil_div(T, 256), 256, 0, st>>>(part, tgt, ids, T, V, nsplit, logp, lse, entropy,
-                                                               status);
+                                                               status, rowmap, n_rows);
   DRK_LAUNCHED();
   return DRK_OK;
 }
@@ -283,7 +291,8 @@ int launch_simt_fwd(const SimtFwdArgs& a, cudaStream_t st) {
                                                                 (const __nv_bfloat16*)a.W, a.ids, a.T, a.H,
                                                                 a.V, per, a.part, a.tgt);
   DRK_LAUNCHED();
-  return launch_lse_merge(a.part, a.tgt, a.ids, a.T, a.V, a.nsplit, a.logp, a.lse, a.entropy, a.status, st);
+  return launch_lse_merge(a.part, a.tgt, a.ids, a.T, a.V, a.nsplit, a.logp, a.lse, a.entropy, a.status, nullptr,
+                          nullptr, st);
 }
 
 template <typename TIn>

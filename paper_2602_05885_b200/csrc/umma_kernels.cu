@@ -222,7 +222,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   int64_t rows = p.rows;
   if (p.n_rows != nullptr) {
     const int cnt = p.n_rows[0];
-    if constexpr (MODE == DL || MODE == DH) {
+    if constexpr (MODE == FWD || MODE == DL || MODE == DH) {
       m_tiles = (cnt + TM * CTAS - 1) / (TM * CTAS);
       rows = p.n_rows[1];
     }
@@ -371,16 +371,16 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       bool row_ok = row < rows;
       // orow: the token this accumulator row belongs to (differs from row when rows are compacted)
       int64_t orow = row;
-      if constexpr (MODE == DL || MODE == DH) {
+      if constexpr (MODE == FWD || MODE == DL || MODE == DH) {
         if (p.rowmap != nullptr) orow = row_ok ? (int64_t)p.rowmap[row] : -1;
-        if constexpr (MODE == DH) row_ok = row_ok && orow >= 0;
+        if constexpr (MODE == DH || MODE == FWD) row_ok = row_ok && orow >= 0;
       }
       // per-unit state
       float run_m = -CUDART_INF_F, run_l = 0.f, run_r = 0.f;  // FWD: log2-domain running max, sum, sum*logit
       int id = -1;
       float c_t = 0.f, z2 = 0.f;
       if constexpr (MODE == FWD) {
-        if (row_ok) id = p.ids[row];
+        if (row_ok) id = p.ids[orow];   // partials and target logits stay indexed by the (compact) row
       }
       if constexpr (MODE == DL) {
         if (row_ok && orow >= 0) { id = p.ids[orow]; c_t = p.coeff[orow]; z2 = p.lse[orow] * kLog2e; }
@@ -639,7 +639,10 @@ int umma_nsplit(int64_t T, int V, int ctas) {
 int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st) {
   const int ctas = a.ctas == 2 ? 2 : 1;
   CUtensorMap mh, mw;
-  if (!make_map(&mh, a.hidden, a.H, a.T, a.H, TK, TM)) return DRK_ERR_CUDA;
+  // With a row map the forward runs over the gathered rows (hidden_c) only; the kernels read their number.
+  const void* hid = a.rowmap ? (const void*)a.hidden_c : a.hidden;
+  const int64_t hid_rows = a.rowmap ? ceil_div(a.T, 256) * 256 : a.T;
+  if (!make_map(&mh, hid, a.H, hid_rows, a.H, TK, TM)) return DRK_ERR_CUDA;
   if (!make_map(&mw, a.W, a.H, a.V, a.H, TK, TN / ctas)) return DRK_ERR_CUDA;
   UmmaParams p{};
   p.m_tiles = (int)ceil_div(a.T, TM * ctas);
@@ -652,9 +655,11 @@ int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st) {
   p.rows = a.T; p.cols = a.V; p.v0 = 0; p.T = a.T;
   p.ids = a.ids; p.part = a.part; p.tgt = a.tgt; p.status = a.status;
   p.want_entropy = a.entropy != nullptr;
+  p.rowmap = a.rowmap; p.n_rows = a.n_rows;
   int rc = launch_mode<FWD>(ctas, mh, mw, p, st);
   if (rc != DRK_OK) return rc;
-  return launch_lse_merge(a.part, a.tgt, a.ids, a.T, a.V, a.nsplit, a.logp, a.lse, a.entropy, a.status, st);
+  return launch_lse_merge(a.part, a.tgt, a.ids, a.T, a.V, a.nsplit, a.logp, a.lse, a.entropy, a.status, a.rowmap,
+                          a.n_rows, st);
 }
 
 int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {

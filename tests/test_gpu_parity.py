@@ -7,6 +7,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import drk_oracle as O
 from paper_2602_05885_b200 import binding as B
 from tests import helpers as Hh
 from tests.gpu_utils import make_params, run_device
@@ -135,3 +136,29 @@ def test_keep_flags_from_the_caller():
     assert Hh.rel_fro(Hh.f64(dev["dW"]), ref["dW"]) <= Hh.TOL_GRAD_FRO
     # seg_w is still this micro-batch's geometric-mean ratio
     assert np.abs(Hh.f64(dev["seg_w"]) - ref["mrs"].w).max() <= 2 * Hh.TOL_LOGP_BF16
+
+
+@pytest.mark.parametrize("engine", [B.DRK_ENGINE_AUTO, B.DRK_ENGINE_UMMA_1CTA])
+def test_forward_over_usable_rows_only(engine):
+    # ragged case: 40 % context tokens and padding in front and behind; their rows are not evaluated
+    case = get_case("ragged")
+    lo, hi = Hh.wide_band(case)
+    veto = PAPER[2]
+    dev = run_device(case, make_params(lo, hi, veto, engine=engine, forward_rows=1))
+    assert dev["status"] == 0
+    need = np.zeros(case.T, dtype=bool)
+    cu = case.cu.numpy()
+    for j in range(case.S):
+        need[cu[j]:cu[j + 1]] = True
+    need &= case.loss_mask.numpy().astype(bool)
+    assert 0 < need.sum() < case.T
+    for k, ref in (("logp", case.logp), ("lse", case.lse), ("entropy", O.token_entropy(case.s))):
+        got = Hh.f64(dev[k])
+        assert np.abs(got[need] - ref[need]).max() <= Hh.TOL_LOGP_BF16, k
+        assert (got[~need] == 0).all(), k
+    # everything downstream only ever reads the usable rows: same decisions, loss and gradients
+    full = dict(dev)
+    for k, ref in (("logp", case.logp), ("lse", case.lse)):
+        full[k] = torch.where(torch.from_numpy(need), dev[k], torch.from_numpy(ref).float())
+    del full["entropy"]
+    Hh.check_against_oracle(case, full, lo, hi, veto)
