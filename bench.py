@@ -344,8 +344,8 @@ def main():
     flops = (2.0 * Tf + 6.0 * Tc) * H * V
     peaks = measured_peaks()
     achieved = flops / (fused_ms * 1e-3) / 1e12
-    # DRAM bytes of one fused call from the committed one-pass ncu capture of exactly this configuration
-    # (profiles/umma_gemm_kernel_pairs_T32768_onepass.md); unknown for any other configuration.
+    # DRAM bytes (read + write) of one fused call, from a one-pass ncu capture of exactly this configuration
+    # with the kernels as they are; unknown (null) for any other configuration.
     traffic = None
     if (args.workload, T, args.mrs, args.dw_dtype, args.dh_dtype, args.v_chunk, args.engine, args.forward_rows) == \
             ("qwen3-14b", 32768, "wide", "f32", "bf16", 0, "auto", "all"):
