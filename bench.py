@@ -218,6 +218,9 @@ def main():
     ap.add_argument("--v-chunk", type=int, default=0)
     ap.add_argument("--forward-rows", default="all", choices=["all", "usable"],
                     help="usable: the forward skips rows that are not loss-masked tokens of a segment")
+    ap.add_argument("--sync-dw", action="store_true",
+                    help="all-reduce dW across ranks slice by slice as the backward finishes each vocabulary chunk "
+                         "(overlapped on a second stream); off by default: the loss path itself needs no collective")
     ap.add_argument("--engine", default="auto", choices=["auto", "1cta"],
                     help="auto: tcgen05 kernels on CTA pairs; 1cta: one CTA per tile")
     ap.add_argument("--mrs", default="wide", choices=["wide", "paper", "off"])
@@ -273,6 +276,15 @@ def main():
     seg_flat = (wl.seg_rollout * Tmax + wl.seg_turn).contiguous()
     stream = torch.cuda.current_stream()
     launches = [0]
+    comm = None
+    if args.sync_dw:
+        # one event per vocabulary chunk; the communication stream reduces a slice of dW once its event fired
+        n_chunks, vc = B.drk_pg_bwd_chunks(T, H, V, code, p)
+        events = [torch.cuda.Event() for _ in range(n_chunks)]
+        for e in events:
+            e.record(stream)
+        B.set_dw_chunk_events(p, [e.cuda_event for e in events])
+        comm = torch.cuda.Stream()
 
     def step(hidden, ids, rl, mask, cu):
         B.drk_trloo_advantage(wl.reward, wl.valid, wl.prompt_of_rollout, R, Tmax, 1.0, B.DRK_BASELINE_TRLOO,
@@ -283,6 +295,9 @@ def main():
                               bufs.lse, bufs.entropy, bufs.seg_w, bufs.seg_keep, bufs.counters, bufs.dH, bufs.dW,
                               bufs.workspace, bufs.workspace_bytes, bufs.status, stream)
         launches[0] += B.drk_last_launch_count()
+        if comm is not None:
+            dp.all_reduce_dw_slices(bufs.dW, vc, events, comm)
+            stream.wait_stream(comm)        # the step ends when the last slice has been reduced
 
     def barrier():
         if world > 1:
@@ -413,7 +428,9 @@ def main():
                        "dW": args.dw_dtype, "dH": args.dh_dtype, "v_chunk": args.v_chunk or "default",
                        "engine": args.engine, "forward_rows": args.forward_rows,
                        "l2": "inputs exceed L2 (W alone is %.2f GB); no flush" % (V * H * 2 / 1e9),
-                       "parallelism": f"dp{world}: one micro-batch per rank, no collective on the loss path"},
+                       "parallelism": f"dp{world}: one micro-batch per rank, " +
+                                      ("dW all-reduced per vocabulary chunk, overlapped" if args.sync_dw
+                                       else "no collective on the loss path")},
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s",
                          "frac": achieved / peaks["tflops"], "traffic": traffic,
                          "kernel": "umma_gemm_kernel (all four instantiations inside one drk_pg_loss_fwd_bwd call)",

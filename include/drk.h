@@ -136,9 +136,24 @@ typedef struct {
                             tokens inside segments); logp, lse, entropy of every other row read 0.  Saves the
                             forward's work on prompt / feedback / padding tokens; tensor-core path only
                             (ignored by the FFMA path)                                                  */
+  void* const* dw_chunk_events; /* NULL, or a host array of n_dw_chunk_events cudaEvent_t: event i is recorded
+                            on the call's stream as soon as rows [i*vc, min(V,(i+1)*vc)) of dW are final, vc and
+                            the chunk count as returned by drk_pg_bwd_chunks().  A data-parallel trainer can
+                            wait on them from a communication stream and start reducing finished slices of dW
+                            while later chunks are still being computed (the gradient exchange itself is the
+                            trainer's; this library makes no collective call)                            */
+  int32_t n_dw_chunk_events; /* must equal the chunk count when dw_chunk_events is given                    */
 } drk_pg_params;
 
 void drk_pg_params_default(drk_pg_params* p); /* host pointer */
+
+/*
+ * How the backward of drk_pg_loss_fwd_bwd walks the vocabulary for these sizes: returns the number of
+ * chunks (>= 1) and stores the chunk width in *v_chunk (every chunk but the last has that many rows of
+ * dW).  Negative drk_status for invalid arguments.  p may be NULL for defaults.
+ */
+int drk_pg_bwd_chunks(int64_t T, int32_t H, int32_t V, int32_t in_dtype, const drk_pg_params* p,
+                      int32_t* v_chunk);
 
 /*
  * Bytes of device workspace needed by drk_pg_logprob_fwd (which = 0) or

@@ -53,6 +53,8 @@ class drk_pg_params(ctypes.Structure):
         ("v_chunk", ctypes.c_int32),
         ("keep_from_caller", ctypes.c_int32),
         ("forward_rows", ctypes.c_int32),
+        ("dw_chunk_events", ctypes.POINTER(ctypes.c_void_p)),
+        ("n_dw_chunk_events", ctypes.c_int32),
     ]
 
 
@@ -98,6 +100,8 @@ def load() -> ctypes.CDLL:
     vp, i32, i64, f32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_size_t
     lib.drk_pg_params_default.argtypes = [ctypes.POINTER(drk_pg_params)]
     lib.drk_pg_params_default.restype = None
+    lib.drk_pg_bwd_chunks.argtypes = [i64, i32, i32, i32, ctypes.POINTER(drk_pg_params), ctypes.POINTER(ctypes.c_int32)]
+    lib.drk_pg_bwd_chunks.restype = ctypes.c_int
     lib.drk_pg_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, ctypes.POINTER(drk_pg_params), i32]
     lib.drk_pg_workspace_bytes.restype = sz
     lib.drk_trloo_advantage.argtypes = [vp, vp, vp, i32, i32, f32, i32, vp, vp, vp, vp]
@@ -167,6 +171,23 @@ def drk_pg_params_default() -> drk_pg_params:
     p = drk_pg_params()
     load().drk_pg_params_default(ctypes.byref(p))
     return p
+
+
+def drk_pg_bwd_chunks(T: int, H: int, V: int, in_dtype: int, p: Optional[drk_pg_params]):
+    """Returns (number of vocabulary chunks of the backward, chunk width)."""
+    vc = ctypes.c_int32(0)
+    n = load().drk_pg_bwd_chunks(T, H, V, in_dtype, ctypes.byref(p) if p is not None else None, ctypes.byref(vc))
+    if n < 0:
+        raise DrkError(n, "drk_pg_bwd_chunks")
+    return n, int(vc.value)
+
+
+def set_dw_chunk_events(p: drk_pg_params, handles) -> None:
+    """Stores raw cudaEvent_t handles (ints) in p; the array is kept alive on p."""
+    arr = (ctypes.c_void_p * len(handles))(*handles)
+    p._dw_event_array = arr
+    p.dw_chunk_events = ctypes.cast(arr, ctypes.POINTER(ctypes.c_void_p))
+    p.n_dw_chunk_events = len(handles)
 
 
 def drk_pg_workspace_bytes(T: int, H: int, V: int, S: int, in_dtype: int,

@@ -131,6 +131,7 @@ bool params_ok(const drk_pg_params& p) {
   if (p.v_chunk < 0) return false;
   if (p.keep_from_caller != 0 && p.keep_from_caller != 1) return false;
   if (p.forward_rows != 0 && p.forward_rows != 1) return false;
+  if (p.n_dw_chunk_events < 0 || (p.dw_chunk_events == nullptr && p.n_dw_chunk_events != 0)) return false;
   if (std::isnan(p.mrs_lo) || std::isnan(p.mrs_hi) || std::isnan(p.veto_ratio)) return false;
   if (p.norm == DRK_NORM_EXPLICIT && !std::isfinite(p.explicit_scale)) return false;
   return true;
@@ -170,6 +171,17 @@ void drk_pg_params_default(drk_pg_params* p) {
   p->v_chunk = 0;
   p->keep_from_caller = 0;
   p->forward_rows = 0;
+  p->dw_chunk_events = nullptr;
+  p->n_dw_chunk_events = 0;
+}
+
+int drk_pg_bwd_chunks(int64_t T, int32_t H, int32_t V, int32_t in_dtype, const drk_pg_params* pp, int32_t* v_chunk) {
+  drk_pg_params p;
+  if (pp) p = *pp; else drk_pg_params_default(&p);
+  if (!sizes_ok(T, H, V, in_dtype) || !params_ok(p) || !v_chunk) return DRK_ERR_INVALID_ARG;
+  const int vc = round_vchunk(p.v_chunk, T, H, V, use_simt(in_dtype, p.engine));
+  *v_chunk = vc;
+  return (int)ceil_div(V, vc);
 }
 
 size_t drk_pg_workspace_bytes(int64_t T, int32_t H, int32_t V, int32_t S, int32_t in_dtype,
@@ -246,6 +258,12 @@ int drk_pg_loss_fwd_bwd(const void* hidden, const void* W, int32_t in_dtype, con
   const bool simt = use_simt(in_dtype, p.engine);
   if (!simt && (H % 8) != 0) return DRK_ERR_UNSUPPORTED;
   if (workspace_bytes < drk_pg_workspace_bytes(T, H, V, S, in_dtype, &p, 1)) return DRK_ERR_WORKSPACE;
+  if (p.dw_chunk_events != nullptr) {
+    const int vc = round_vchunk(p.v_chunk, T, H, V, simt);
+    if (T == 0 || p.n_dw_chunk_events != (int)ceil_div(V, vc)) return DRK_ERR_INVALID_ARG;
+    for (int i = 0; i < p.n_dw_chunk_events; ++i)
+      if (p.dw_chunk_events[i] == nullptr) return DRK_ERR_INVALID_ARG;
+  }
   int rc = check_arch();
   if (rc != DRK_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -297,7 +315,7 @@ int drk_pg_loss_fwd_bwd(const void* hidden, const void* W, int32_t in_dtype, con
   }
   if (simt) {
     SimtBwdArgs b{hidden, W, in_dtype, ids, T, H, V, lse, bw.coeff, static_cast<float*>(bw.dL), bw.vc,
-                  dH, p.dh_dtype, bw.dH_acc, dW, p.dw_dtype, p.dw_accumulate};
+                  dH, p.dh_dtype, bw.dH_acc, dW, p.dw_dtype, p.dw_accumulate, p.dw_chunk_events};
     rc = launch_simt_bwd(b, st);
   } else {
     CompactArgs ca{bw.coeff, static_cast<const __nv_bfloat16*>(hidden), T, H, bw.blk_cnt, bw.blk_off, bw.n_rows,
@@ -306,7 +324,7 @@ int drk_pg_loss_fwd_bwd(const void* hidden, const void* W, int32_t in_dtype, con
     if (rc != DRK_OK) return fail(rc);
     UmmaBwdArgs b{hidden, W, ids, T, H, V, lse, bw.coeff, static_cast<__nv_bfloat16*>(bw.dL), bw.vc,
                   dH, p.dh_dtype, bw.dH_acc, dW, p.dw_dtype, p.dw_accumulate, status, umma_ctas(p.engine),
-                  bw.hidden_c, bw.rowmap, bw.n_rows};
+                  bw.hidden_c, bw.rowmap, bw.n_rows, p.dw_chunk_events};
     rc = launch_umma_bwd(b, st);
   }
   if (rc != DRK_OK) return fail(rc);

@@ -62,6 +62,7 @@ struct SimtBwdArgs {
   const float* lse; const float* coeff; float* dL /*[T*vc] fp32 workspace*/; int vc;
   void* dH; int dh_dtype; float* dH_acc /*fp32 [T,H] or null when dH is fp32*/;
   void* dW; int dw_dtype; int dw_accumulate;
+  void* const* chunk_events;  // optional cudaEvent_t per vocabulary chunk, recorded when its dW rows are final
 };
 int launch_simt_bwd(const SimtBwdArgs& a, cudaStream_t st);
 
@@ -82,6 +83,7 @@ struct UmmaBwdArgs {
   void* dH; int dh_dtype; float* dH_acc; void* dW; int dw_dtype; int dw_accumulate; uint32_t* status;
   int ctas;
   const __nv_bfloat16* hidden_c; const int32_t* rowmap; const int32_t* n_rows;  // compacted rows
+  void* const* chunk_events;  // optional cudaEvent_t per vocabulary chunk, recorded when its dW rows are final
 };
 int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st);
 

@@ -317,6 +317,7 @@ static int simt_bwd_typed(const SimtBwdArgs& a, cudaStream_t st) {
                                                                (__nv_bfloat16*)a.dW + (int64_t)v0 * a.H, a.H,
                                                                vc_this, a.H, a.T, a.dw_accumulate);
     DRK_LAUNCHED();
+    if (a.chunk_events != nullptr) DRK_CUDA_CHECK(cudaEventRecord(static_cast<cudaEvent_t>(a.chunk_events[chunk]), st));
     // dH (+)= dL W[v0:v0+vc_this, :]              (M = t, N = h, K = v)
     dim3 g3((unsigned)ceil_div(a.T, BM), (unsigned)ceil_div(a.H, BN));
     gemm_kernel<TIn, float><<<g3, kThreads, 0, st>>>(a.dL, a.vc, 1, W + (int64_t)v0 * a.H, a.H, 1, dh_acc, a.H, a.T,

@@ -709,6 +709,8 @@ int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {
       p.rowmap = a.rowmap; p.n_rows = a.n_rows;
       int rc = launch_mode<DW>(ctas, mdl_mn, mh_mn, p, st);
       if (rc != DRK_OK) return rc;
+      if (a.chunk_events != nullptr)
+        DRK_CUDA_CHECK(cudaEventRecord(static_cast<cudaEvent_t>(a.chunk_events[chunk]), st));
     }
     {  // dH (+)= dL W[v0 : v0 + vc_this, :]
       UmmaParams p{};

@@ -36,3 +36,31 @@ def sum_over_ranks(value: float, device="cpu") -> float:
     t = torch.tensor([float(value)], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.SUM)
     return float(t.item())
+
+
+def chunk_slices(V: int, v_chunk: int):
+    """Row ranges [a, b) of dW that the backward finishes one after the other."""
+    return [(a, min(V, a + v_chunk)) for a in range(0, V, v_chunk)]
+
+
+def all_reduce_dw_slices(dW: torch.Tensor, v_chunk: int, events=None, comm_stream=None):
+    """Sums dW over the ranks slice by slice, in the order in which the backward finishes the slices.
+
+    On a GPU, `events[i]` (recorded by the library when slice i is final) gates slice i on `comm_stream`,
+    so the reduction of early slices overlaps the computation of later ones.  Without events (CPU tensors,
+    gloo) the slices are reduced one after the other.  Returns the number of slices.
+    """
+    slices = chunk_slices(dW.shape[0], v_chunk)
+    multi = dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1
+    if events is None:
+        for a, b in slices:
+            if multi:
+                dist.all_reduce(dW[a:b])
+        return len(slices)
+    assert len(events) == len(slices)
+    with torch.cuda.stream(comm_stream):
+        for (a, b), e in zip(slices, events):
+            comm_stream.wait_event(e)
+            if multi:
+                dist.all_reduce(dW[a:b])
+    return len(slices)

@@ -30,6 +30,11 @@ def _worker(rank, world, port, out):
     t_rank = 1.0 + rank            # pretend rank 1 is slower
     t_job = dp.max_over_ranks(t_rank)
     total = dp.sum_over_ranks(tokens)
+    # gradient exchange by vocabulary slices, in the order in which the backward finishes them
+    dW = torch.full((1000, 4), float(rank + 1))
+    n_slices = dp.all_reduce_dw_slices(dW, 256)
+    assert n_slices == 4 and dp.chunk_slices(1000, 256)[-1] == (768, 1000)
+    assert torch.equal(dW, torch.full((1000, 4), 3.0))          # 1 + 2 on every element, every slice covered once
     out.put((rank, mine, tokens, t_job, total, len(plans), sum(p.used for p in plans)))
     dist.destroy_process_group()
 

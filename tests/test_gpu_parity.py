@@ -162,3 +162,39 @@ def test_forward_over_usable_rows_only(engine):
         full[k] = torch.where(torch.from_numpy(need), dev[k], torch.from_numpy(ref).float())
     del full["entropy"]
     Hh.check_against_oracle(case, full, lo, hi, veto)
+
+
+def test_dw_chunk_events_mark_finished_slices():
+    # a communication stream may start on a slice of dW as soon as its event has fired
+    case = get_case("medium")
+    d = torch.device("cuda:0")
+    p = make_params(0.0, math.inf, 0.0, v_chunk=2048)
+    n_chunks, vc = B.drk_pg_bwd_chunks(case.T, case.H, case.V, B.DRK_BF16, p)
+    assert vc == 2048 and n_chunks == math.ceil(case.V / 2048) > 1
+    events = [torch.cuda.Event() for _ in range(n_chunks)]
+    for e in events:
+        e.record()                      # creates the underlying cudaEvent_t
+    B.set_dw_chunk_events(p, [e.cuda_event for e in events])
+    bufs = B.PgLossBuffers(case.T, case.H, case.V, case.S, B.DRK_BF16, p, d)
+    bufs.dW.fill_(float("nan"))
+    snap = torch.zeros_like(bufs.dW)
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    B.pg_loss_fwd_bwd(case.hidden.to(d), case.W.to(d), case.ids.to(d), case.rollout_logp.to(d), case.loss_mask.to(d),
+                      case.cu.to(d), case.seg_adv.to(d), p, bufs)
+    with torch.cuda.stream(side):
+        for i, e in enumerate(events):
+            side.wait_event(e)
+            a, b = i * vc, min(case.V, (i + 1) * vc)
+            snap[a:b].copy_(bufs.dW[a:b], non_blocking=True)
+    torch.cuda.synchronize()
+    assert torch.isfinite(snap).all() and torch.equal(snap, bufs.dW)
+    ref = Hh.oracle_eval(case, 0.0, math.inf, 0.0)
+    assert Hh.rel_fro(Hh.f64(bufs.dW), ref["dW"]) <= Hh.TOL_GRAD_FRO
+    # a wrong event count is rejected before anything is enqueued
+    B.set_dw_chunk_events(p, [e.cuda_event for e in events[:-1]])
+    rc = B.drk_pg_loss_fwd_bwd(case.hidden.to(d), case.W.to(d), B.DRK_BF16, case.ids.to(d), case.rollout_logp.to(d),
+                               case.loss_mask.to(d), case.cu.to(d), case.seg_adv.to(d), case.T, case.H, case.V, case.S,
+                               p, bufs.loss, bufs.logp, bufs.lse, None, bufs.seg_w, bufs.seg_keep, bufs.counters,
+                               bufs.dH, bufs.dW, bufs.workspace, bufs.workspace_bytes, bufs.status, check=False)
+    assert rc == B.DRK_ERR_INVALID_ARG
