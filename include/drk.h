@@ -193,7 +193,7 @@ int drk_pg_logprob_fwd(const void* hidden, const void* W, int32_t in_dtype, cons
  * packaging variant of the forward call above.)  The scratch (per-row partial max / sum-exp pairs and
  * target logits) lives in a fixed array inside the library image instead:
  *   - every GPU on which the library is loaded holds DRK_NOALLOC_SCRATCH_BYTES until the process exits;
- *   - if the sizes need more (roughly 16*nsplit*T + 4*T bytes, nsplit <= 32 chosen from T, H and V) the call
+ *   - if the sizes need more (roughly 16*nsplit*T + 4*T bytes, nsplit <= 32 chosen from T and V) the call
  *     returns DRK_ERR_WORKSPACE and enqueues nothing; T = 32768 at H = 5120, V = 151936 needs about 2.2 MB;
  *   - the array is shared by all calls on a device and keeps the last call's contents.  What the
  *     computation reads is rewritten or cleared by each call, so consecutive calls on one stream are

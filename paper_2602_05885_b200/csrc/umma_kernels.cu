@@ -615,25 +615,31 @@ int launch_mode(int ctas, const CUtensorMap& a, const CUtensorMap& b, const Umma
 
 }  // namespace
 
+// Number of vocabulary ranges per row tile in the forward: work units (row tile, range) should fill
+// whole waves of the resident CTAs (or pairs).  Among the counts within 1 % of the best wave
+// efficiency the smallest is taken: fewer partials to write and merge, and measured call times do
+// not distinguish them.
 int umma_nsplit(int64_t T, int V, int ctas) {
   const int64_t m_tiles = ceil_div(T, TM * ctas);
   const int n_tiles = (int)ceil_div(V, TN);
   if (m_tiles <= 0) return 1;
   const int sms = 148 / ctas;
-  int best = 1;
+  double eff[33];
   double best_eff = -1.0;
-  for (int ns = 1; ns <= 32 && ns <= n_tiles; ++ns) {
+  for (int ns = 1; ns <= 32; ++ns) {
+    eff[ns] = -1.0;
+    if (ns > n_tiles) continue;
     const int per = (int)ceil_div(n_tiles, ns);
-    const int ns_eff = (int)ceil_div(n_tiles, per);
-    if (ns_eff != ns) continue;
+    if ((int)ceil_div(n_tiles, per) != ns) continue;
     if (per < 4 && ns > 1) continue;
-    const int64_t units = m_tiles * ns;
-    const int64_t waves = ceil_div(units, sms);
+    const int64_t waves = ceil_div(m_tiles * ns, sms);
     // time ~ waves * per tiles; work = m_tiles * n_tiles tiles
-    const double eff = (double)(m_tiles * (int64_t)n_tiles) / ((double)waves * per * sms);
-    if (eff > best_eff + 0.005) { best_eff = eff; best = ns; }
+    eff[ns] = (double)(m_tiles * (int64_t)n_tiles) / ((double)waves * per * sms);
+    if (eff[ns] > best_eff) best_eff = eff[ns];
   }
-  return best;
+  for (int ns = 1; ns <= 32; ++ns)
+    if (eff[ns] >= best_eff - 0.01) return ns;
+  return 1;
 }
 
 int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st) {

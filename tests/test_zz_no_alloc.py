@@ -71,3 +71,5 @@ def test_sizes_beyond_the_fixed_scratch_are_rejected():
     assert rc == B.DRK_ERR_WORKSPACE
     assert B.drk_last_launch_count() == 0
     assert "workspace" in B.drk_status_string(rc)
+    # the 14B training shape fits the fixed array with room to spare
+    assert B.drk_pg_workspace_bytes(32768, 5120, 151936, 0, B.DRK_BF16, None, 0) < B.DRK_NOALLOC_SCRATCH_BYTES // 2
