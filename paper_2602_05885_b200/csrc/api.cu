@@ -83,7 +83,7 @@ struct FwdWs {
 };
 FwdWs carve_fwd(Carver& c, int64_t T, int V, bool simt, int engine) {
   FwdWs w;
-  w.nsplit = simt ? simt_nsplit(T, V) : umma_nsplit(T, V, umma_ctas(engine));
+  w.nsplit = simt ? simt_nsplit(T, V) : umma_nsplit(T, V, umma_ctas(engine), false);
   w.part = static_cast<float*>(c.take(sizeof(float) * 4 * (size_t)w.nsplit * (size_t)T));
   w.tgt = static_cast<float*>(c.take(sizeof(float) * (size_t)T));
   return w;

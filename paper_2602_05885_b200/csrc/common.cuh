@@ -75,7 +75,7 @@ struct UmmaFwdArgs {
   // optional: evaluate only the rows listed in rowmap (gathered into hidden_c); others are left untouched
   const __nv_bfloat16* hidden_c; const int32_t* rowmap; const int32_t* n_rows;
 };
-int umma_nsplit(int64_t T, int V, int ctas);
+int umma_nsplit(int64_t T, int V, int ctas, bool frugal);
 int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st);
 struct UmmaBwdArgs {
   const void* hidden; const void* W; const int32_t* ids; int64_t T; int H; int V;

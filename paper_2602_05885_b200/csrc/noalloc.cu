@@ -72,7 +72,7 @@ extern "C" int drk_pg_logprob_fwd_noalloc(const void* hidden, const void* W, int
 
   // scratch layout: partials [nsplit, T, 4] floats, then target logits [T] floats, each 256-aligned
   const int ctas = engine == DRK_ENGINE_UMMA_1CTA ? 1 : 2;
-  const int nsplit = simt ? simt_nsplit(T, V) : umma_nsplit(T, V, ctas);
+  const int nsplit = simt ? simt_nsplit(T, V) : umma_nsplit(T, V, ctas, true);
   const size_t part_bytes = align_up(sizeof(float) * 4 * (size_t)nsplit * (size_t)T, 256);
   const size_t tgt_bytes = align_up(sizeof(float) * (size_t)T, 256);
   if (part_bytes + tgt_bytes > kScratchBytes) return DRK_ERR_WORKSPACE;
