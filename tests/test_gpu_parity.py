@@ -198,3 +198,15 @@ def test_dw_chunk_events_mark_finished_slices():
                                p, bufs.loss, bufs.logp, bufs.lse, None, bufs.seg_w, bufs.seg_keep, bufs.counters,
                                bufs.dH, bufs.dW, bufs.workspace, bufs.workspace_bytes, bufs.status, check=False)
     assert rc == B.DRK_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("engine", [B.DRK_ENGINE_AUTO, B.DRK_ENGINE_UMMA_1CTA])
+def test_results_are_reproducible_bit_for_bit(engine):
+    # no atomics on the loss path: two calls on the same inputs give identical bits
+    case = get_case("medium")
+    lo, hi = Hh.wide_band(case)
+    p = make_params(lo, hi, PAPER[2], engine=engine, v_chunk=2048, dh_dtype=B.DRK_BF16)
+    a = run_device(case, p)
+    b = run_device(case, p)
+    for k in ("logp", "lse", "entropy", "seg_w", "seg_keep", "loss", "counters", "dH", "dW"):
+        assert torch.equal(a[k], b[k]), k
