@@ -286,14 +286,15 @@ def main():
         B.set_dw_chunk_events(p, [e.cuda_event for e in events])
         comm = torch.cuda.Stream()
 
-    def step(hidden, ids, rl, mask, cu):
+    def step(hidden, ids, rl, mask, cu, out=None):
+        o = out if out is not None else bufs
         B.drk_trloo_advantage(wl.reward, wl.valid, wl.prompt_of_rollout, R, Tmax, 1.0, B.DRK_BASELINE_TRLOO,
                               ret, adv, gsize, stream)
         launches[0] += B.drk_last_launch_count()
         seg_adv = adv.view(-1).index_select(0, seg_flat)     # the caller's gather of per-sample advantages
-        B.drk_pg_loss_fwd_bwd(hidden, wl.W, code, ids, rl, mask, cu, seg_adv, T, H, V, S, p, bufs.loss, bufs.logp,
-                              bufs.lse, bufs.entropy, bufs.seg_w, bufs.seg_keep, bufs.counters, bufs.dH, bufs.dW,
-                              bufs.workspace, bufs.workspace_bytes, bufs.status, stream)
+        B.drk_pg_loss_fwd_bwd(hidden, wl.W, code, ids, rl, mask, cu, seg_adv, T, H, V, S, p, o.loss, o.logp,
+                              o.lse, o.entropy, o.seg_w, o.seg_keep, o.counters, o.dH, o.dW,
+                              o.workspace, o.workspace_bytes, o.status, stream)
         launches[0] += B.drk_last_launch_count()
         if comm is not None:
             dp.all_reduce_dw_slices(bufs.dW, vc, events, comm)
@@ -389,30 +390,64 @@ def main():
         h2d = sum(t.numel() * t.element_size() for t in host)
         d2h = sum(t.numel() * t.element_size() for t in (h_loss, h_cnt, h_logp, h_keep, h_dH))
 
-        def e2e_step():
-            for src, dst in zip(host, devin):
-                dst.copy_(src, non_blocking=True)
-            step(*devin)
-            h_loss.copy_(bufs.loss, non_blocking=True)
-            h_cnt.copy_(bufs.counters, non_blocking=True)
-            h_logp.copy_(bufs.logp, non_blocking=True)
-            h_keep.copy_(bufs.seg_keep, non_blocking=True)
-            h_dH.copy_(bufs.dH, non_blocking=True)
+        # Two sets of device inputs and outputs: the upload of step i+1 and the download of step i-1 run on
+        # their own streams while step i computes, as a trainer's input pipeline would do.  Every step still
+        # moves its own inputs in and its own results out inside the timed region.
+        bufs2 = B.PgLossBuffers(T, H, V, S, code, p, dev, dW=bufs.dW)
+        out_sets = [bufs, bufs2]
+        in_sets = [devin, [torch.empty_like(t, device=dev) for t in host]]
+        up, down = torch.cuda.Stream(), torch.cuda.Stream()
+        ev_up = [torch.cuda.Event() for _ in range(2)]
+        ev_done = [torch.cuda.Event() for _ in range(2)]
+        ev_down = [torch.cuda.Event() for _ in range(2)]
 
-        for _ in range(2):
-            e2e_step()
+        def upload(k):
+            with torch.cuda.stream(up):
+                up.wait_event(ev_done[k])                 # the step that last read this input set has finished
+                for src, dst in zip(host, in_sets[k]):
+                    dst.copy_(src, non_blocking=True)
+                ev_up[k].record(up)
+
+        def download(k):
+            with torch.cuda.stream(down):
+                down.wait_event(ev_done[k])
+                o = out_sets[k]
+                h_loss.copy_(o.loss, non_blocking=True)
+                h_cnt.copy_(o.counters, non_blocking=True)
+                h_logp.copy_(o.logp, non_blocking=True)
+                h_keep.copy_(o.seg_keep, non_blocking=True)
+                h_dH.copy_(o.dH, non_blocking=True)
+                ev_down[k].record(down)
+
+        def e2e_run(n):
+            for k in range(2):
+                ev_done[k].record(stream)
+                ev_down[k].record(stream)
+            upload(0)
+            for i in range(n):
+                k = i % 2
+                stream.wait_event(ev_up[k])               # this step's inputs have arrived
+                stream.wait_event(ev_down[k])             # this output set has been read back (two steps ago)
+                step(*in_sets[k], out=out_sets[k])
+                ev_done[k].record(stream)
+                if i + 1 < n:
+                    upload(1 - k)
+                download(k)
+            stream.wait_stream(down)
+
+        e2e_run(2)
         barrier()
-        t0 = time.perf_counter()
         ev0.record(stream)
-        for _ in range(args.steps):
-            e2e_step()
+        e2e_run(args.steps)
         ev1.record(stream)
         barrier()
         e_ms = dp.max_over_ranks(ev0.elapsed_time(ev1), dev)
         e2e = {"value": world * T * args.steps / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": e_ms / args.steps,
-               "what": "hidden, ids, rollout log-probs, mask, cu_seqlens copied from pinned host memory each step; "
-                       "loss, counters, log-probs, keep flags and dH copied back; W and dW stay resident"}
+               "what": "every step: hidden, ids, rollout log-probs, mask, cu_seqlens copied from pinned host memory; "
+                       "loss, counters, log-probs, keep flags and dH copied back to pinned host memory; uploads and "
+                       "downloads run on their own streams, double-buffered against the compute; W and dW stay "
+                       "resident"}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
