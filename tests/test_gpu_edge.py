@@ -107,3 +107,31 @@ def test_host_detected_errors_return_codes():
     torch.cuda.synchronize()
     assert torch.allclose(logp, torch.full_like(logp, -math.log(V)), atol=1e-5)
     assert B.drk_last_launch_count() == 2
+
+
+@pytest.mark.parametrize("T,H,V", [(1, 64, 300), (129, 72, 4099), (300, 512, 257)])
+def test_forward_over_usable_rows_at_ragged_sizes(T, H, V):
+    case = Hh.build_plain_case(f"fr{T}", T=T, H=H, V=V, dtype=torch.bfloat16, S=3, seed=T + V + 1, mask_frac=0.3)
+    dev = run_device(case, make_params(*OPEN, v_chunk=256, forward_rows=1))
+    assert dev["status"] == 0
+    need = case.loss_mask.numpy().astype(bool)
+    got = Hh.f64(dev["logp"])
+    if need.any():
+        assert np.abs(got[need] - case.logp[need]).max() <= Hh.TOL_LOGP_BF16
+    assert (got[~need] == 0).all()
+    full = dict(dev)
+    full["logp"] = torch.where(torch.from_numpy(need), dev["logp"], torch.from_numpy(case.logp).float())
+    full["lse"] = torch.where(torch.from_numpy(need), dev["lse"], torch.from_numpy(case.lse).float())
+    del full["entropy"]
+    Hh.check_against_oracle(case, full, *OPEN)
+
+
+def test_forward_rows_with_nothing_usable():
+    # every token masked out: no row is evaluated, nothing is retained, gradients are exactly zero
+    case = Hh.build_plain_case("fr0", T=200, H=64, V=700, dtype=torch.bfloat16, S=2, seed=77)
+    case.loss_mask = torch.zeros_like(case.loss_mask)
+    dev = run_device(case, make_params(*OPEN, forward_rows=1))
+    assert dev["status"] == 0
+    assert (dev["logp"] == 0).all() and (dev["lse"] == 0).all() and (dev["entropy"] == 0).all()
+    assert (dev["seg_keep"] == 0).all() and (dev["counters"] == 0).all() and float(dev["loss"]) == 0.0
+    assert (dev["dH"] == 0).all() and (dev["dW"] == 0).all()
