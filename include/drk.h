@@ -131,7 +131,10 @@ typedef struct {
                             the caller has already decided which samples are retained (e.g. a sample
                             split over several micro-batches, judged on log-probs from
                             drk_pg_logprob_fwd of all its pieces); seg_w and the counters are still
-                            computed from this micro-batch's tokens                                   */
+                            computed from this micro-batch's tokens.  2: seg_keep holds the caller's
+                            retention flags on input (for instance `retain` of drk_reward, i.e. the
+                            profiling-based rejection sampling of Sec. 5.2) and a sample is kept iff its
+                            flag is set AND it passes the MRS test; seg_keep returns the combined decision */
   int32_t forward_rows;  /* 0: log-probs of all T rows.  1: only of the rows the loss can use (loss-masked
                             tokens inside segments); logp, lse, entropy of every other row read 0.  Saves the
                             forward's work on prompt / feedback / padding tokens; tensor-core path only

@@ -129,7 +129,7 @@ bool params_ok(const drk_pg_params& p) {
   if (p.dh_dtype != DRK_F32 && p.dh_dtype != DRK_BF16) return false;
   if (!engine_ok(p.engine)) return false;
   if (p.v_chunk < 0) return false;
-  if (p.keep_from_caller != 0 && p.keep_from_caller != 1) return false;
+  if (p.keep_from_caller < 0 || p.keep_from_caller > 2) return false;
   if (p.forward_rows != 0 && p.forward_rows != 1) return false;
   if (p.n_dw_chunk_events < 0 || (p.dw_chunk_events == nullptr && p.n_dw_chunk_events != 0)) return false;
   if (std::isnan(p.mrs_lo) || std::isnan(p.mrs_hi) || std::isnan(p.veto_ratio)) return false;

@@ -116,7 +116,8 @@ finalize_kernel(double* __restrict__ seg_stats, const float* __restrict__ seg_ad
       w = (float)exp(mean);
       vetoed = st[2] < ln_veto;
       keep = (ln_lo <= mean) && (mean <= ln_hi) && !vetoed;
-      if (keep_from_caller) keep = seg_keep[g] != 0;   // the caller's decision stands (never for empty segments)
+      if (keep_from_caller == 1) keep = seg_keep[g] != 0;            // the caller's decision stands
+      else if (keep_from_caller == 2) keep = keep && seg_keep[g] != 0;  // caller's retention AND the MRS test
     }
     seg_w[g] = w;
     seg_keep[g] = keep ? 1 : 0;

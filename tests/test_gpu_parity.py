@@ -210,3 +210,23 @@ def test_results_are_reproducible_bit_for_bit(engine):
     b = run_device(case, p)
     for k in ("logp", "lse", "entropy", "seg_w", "seg_keep", "loss", "counters", "dH", "dW"):
         assert torch.equal(a[k], b[k]), k
+
+
+def test_caller_retention_combined_with_mrs():
+    # PRS-style retention flags from the caller, ANDed with the mismatch rejection decided here
+    case = get_case("medium")
+    lo, hi = Hh.wide_band(case)
+    g = torch.Generator().manual_seed(4)
+    retain = (torch.rand(case.S, generator=g) < 0.7).to(torch.uint8)
+    dev = run_device(case, make_params(lo, hi, PAPER[2], keep_from_caller=2), keep_in=retain)
+    m = Hh.oracle_eval(case, lo, hi, PAPER[2], want_grads=False)["mrs"]
+    amb = Hh.ambiguous_segments(m, lo, hi, PAPER[2], Hh.TOL_LOGP_BF16, Hh.TOL_LOGP_BF16)
+    expect = m.keep & retain.numpy().astype(bool)
+    got = dev["seg_keep"].numpy().astype(bool)
+    assert not ((got != expect) & ~amb).any()
+    assert not (got & ~retain.numpy().astype(bool)).any()          # never kept against the caller's flag
+    assert 0 < got.sum() < m.keep.sum()
+    ref = Hh.oracle_eval(case, lo, hi, PAPER[2], keep_override=got)
+    assert dev["counters"][0] == ref["kept_tokens"] and dev["counters"][2] == ref["kept_segs"]
+    assert Hh.rel_fro(Hh.f64(dev["dH"]), ref["dH"]) <= Hh.TOL_GRAD_FRO
+    assert Hh.rel_fro(Hh.f64(dev["dW"]), ref["dW"]) <= Hh.TOL_GRAD_FRO
