@@ -627,7 +627,14 @@ int umma_nsplit(int64_t T, int V, int ctas, bool frugal) {
   const int64_t m_tiles = ceil_div(T, TM * ctas);
   const int n_tiles = (int)ceil_div(V, TN);
   if (m_tiles <= 0) return 1;
-  if (!frugal) return (int)ceil_div(n_tiles, 2);
+  if (!frugal) {
+    // ranges of two tiles, longer ones where the partials (16 bytes per row and range) would pass 256 MiB
+    int64_t cap = ((int64_t)1 << 28) / (16 * T);
+    if (cap < 32) cap = 32;
+    int64_t per = 2;
+    if (ceil_div(n_tiles, per) > cap) per = ceil_div(n_tiles, cap);
+    return (int)ceil_div(n_tiles, per);
+  }
   const int sms = 148 / ctas;
   double eff[33];
   double best_eff = -1.0;
@@ -669,7 +676,7 @@ int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st) {
   p.nj = a.nsplit;
   p.tiles_per_unit = (int)ceil_div(p.n_tiles, a.nsplit);
   const int slots = 148 / ctas;
-  if (a.nsplit * 8 >= p.n_tiles) p.group_m = panel_group(TM * ctas, a.H);          // short units: panel budget
+  if (a.nsplit > 32 || a.nsplit * 8 >= p.n_tiles) p.group_m = panel_group(TM * ctas, a.H);  // short units: panel budget
   else p.group_m = slots / a.nsplit > 0 ? slots / a.nsplit : 1;                    // long ranges: one wave
   p.rows = a.T; p.cols = a.V; p.v0 = 0; p.T = a.T;
   p.ids = a.ids; p.part = a.part; p.tgt = a.tgt; p.status = a.status;
