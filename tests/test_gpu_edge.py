@@ -135,3 +135,25 @@ def test_forward_rows_with_nothing_usable():
     assert (dev["logp"] == 0).all() and (dev["lse"] == 0).all() and (dev["entropy"] == 0).all()
     assert (dev["seg_keep"] == 0).all() and (dev["counters"] == 0).all() and float(dev["loss"]) == 0.0
     assert (dev["dH"] == 0).all() and (dev["dW"] == 0).all()
+
+
+@pytest.mark.parametrize("engine", [B.DRK_ENGINE_AUTO, B.DRK_ENGINE_SIMT])
+def test_large_logits_stay_finite_and_accurate(engine):
+    # logits of magnitude ~100: the running-max subtraction must keep exp() in range on every tile
+    case = Hh.build_plain_case("big", T=300, H=512, V=5000, dtype=torch.bfloat16, S=3, seed=91)
+    case.hidden = (case.hidden.float() * 8).to(torch.bfloat16)
+    case.W = (case.W.float() * 8).to(torch.bfloat16)
+    from oracle import drk_oracle as O
+    case.s = O.logits(Hh.f64(case.hidden), Hh.f64(case.W))
+    assert np.abs(case.s).max() > 80
+    case.logp, case.lse = O.token_logprob(case.s, case.ids.numpy())
+    case.rollout_logp = torch.from_numpy(case.logp.astype(np.float32))
+    dev = run_device(case, make_params(*OPEN, engine=engine, v_chunk=1024))
+    assert dev["status"] == 0
+    assert torch.isfinite(dev["logp"]).all() and torch.isfinite(dev["dW"]).all() and torch.isfinite(dev["dH"]).all()
+    # fp32 accumulation of ~100-sized logits: absolute error scales with the magnitude
+    tol = Hh.TOL_LOGP_BF16 * max(1.0, float(np.abs(case.logp).max()) / 10)
+    assert np.abs(Hh.f64(dev["logp"]) - case.logp).max() <= tol
+    ref = Hh.oracle_eval(case, *OPEN)
+    assert Hh.rel_fro(Hh.f64(dev["dH"]), ref["dH"]) <= Hh.TOL_GRAD_FRO
+    assert Hh.rel_fro(Hh.f64(dev["dW"]), ref["dW"]) <= Hh.TOL_GRAD_FRO
