@@ -19,6 +19,12 @@ What follows the paper, and where:
   mrs()                geometric mismatch rejection sampling    Sec. 5.1 (unnumbered eq.)
                        with the token-level veto
   coeff_and_loss()     REINFORCE surrogate                      App. A (estimator g-hat)
+  segment_advantages()  advantage of the (rollout, turn) sample    Sec. 4.3 (every turn of a trajectory
+                       a packed segment holds                   is one training sample)
+  shard_stats()/merge_shard_stats()/shard_gradients()
+                       the same definitions restricted to a range of vocabulary columns, and the
+                       exact recombination of such ranges (the paper has no counterpart: this is
+                       what each GPU of a vocabulary-split LM head can know on its own)
   logits()/token_logprob()/gradients()
                        the plain definition of log-softmax over the LM head
                        and its analytic gradient (the paper names the trainer
@@ -122,6 +128,16 @@ def trloo_advantage(G, valid, prompt_of_rollout):
                 others = sum(G[j, t] for j in g if j != i)
                 A[i, t] = G[i, t] - others / (n - 1)
     return A, N
+
+
+def segment_advantages(A, seg_rollout, seg_turn):
+    """Sec. 4.3: each turn of a trajectory is one training sample.  Segment g of a packed micro-batch
+    holds turn seg_turn[g] of rollout seg_rollout[g]; every token of it carries A[seg_rollout[g], seg_turn[g]]."""
+    A = np.asarray(A, dtype=F64)
+    out = np.zeros(len(seg_rollout), dtype=F64)
+    for g in range(len(seg_rollout)):
+        out[g] = A[int(seg_rollout[g]), int(seg_turn[g])]
+    return out
 
 
 # ---------------------------------------------------------------------------
@@ -280,6 +296,53 @@ def gradients(hidden, W, s, lse, ids, coeff):
     dH = np.matmul(dL, np.asarray(W, dtype=F64))
     dW = np.matmul(dL.T, np.asarray(hidden, dtype=F64))
     return dH, dW
+
+
+# ---------------------------------------------------------------------------
+# The same quantities when the vocabulary is split into column ranges (one range per GPU)
+# ---------------------------------------------------------------------------
+
+def shard_stats(s, ids, v_begin, v_end):
+    """What the owner of columns [v_begin, v_end) knows about each row t, from its own logits only:
+    m = max_v s[t,v];  l = sum_v exp(s[t,v] - m);  r = sum_v exp(s[t,v] - m) * s[t,v];
+    g = s[t, ids[t]] if v_begin <= ids[t] < v_end else 0.   Returns an array [T, 4] = (m, l, r, g)."""
+    s = np.asarray(s, dtype=F64)
+    ids = np.asarray(ids, dtype=np.int64)
+    T = s.shape[0]
+    out = np.zeros((T, 4), dtype=F64)
+    for t in range(T):
+        row = s[t, v_begin:v_end]
+        m = row.max()
+        e = np.exp(row - m)
+        out[t, 0] = m
+        out[t, 1] = e.sum()
+        out[t, 2] = (e * row).sum()
+        if v_begin <= ids[t] < v_end:
+            out[t, 3] = s[t, ids[t]]
+    return out
+
+
+def merge_shard_stats(stats):
+    """Recombines shard_stats of ranges that partition the vocabulary (stats: [n, T, 4]):
+    M = max_k m_k;  L = sum_k l_k exp(m_k - M);  lse = M + ln L;  logp = sum_k g_k - lse;
+    entropy = lse - (sum_k r_k exp(m_k - M)) / L.   Returns (logp, lse, entropy)."""
+    st = np.asarray(stats, dtype=F64)
+    M = st[:, :, 0].max(axis=0)
+    wgt = np.exp(st[:, :, 0] - M[None, :])
+    L = (st[:, :, 1] * wgt).sum(axis=0)
+    Rr = (st[:, :, 2] * wgt).sum(axis=0)
+    lse = M + np.log(L)
+    return st[:, :, 3].sum(axis=0) - lse, lse, lse - Rr / L
+
+
+def shard_gradients(hidden, W, s, lse, ids, coeff, v_begin, v_end):
+    """The part of the gradients that the owner of columns [v_begin, v_end) forms from them alone:
+    dH_part[t,:] = sum_{v in range} dL[t,v] W[v,:]  (the ranges' parts add up to dH);
+    dW_rows[v,:] = sum_t dL[t,v] hidden[t,:] for v in the range (rows v_begin..v_end of dW)."""
+    dL = dlogits(s, lse, ids, coeff)[:, v_begin:v_end]
+    dH_part = np.matmul(dL, np.asarray(W, dtype=F64)[v_begin:v_end])
+    dW_rows = np.matmul(dL.T, np.asarray(hidden, dtype=F64))
+    return dH_part, dW_rows
 
 
 # ---------------------------------------------------------------------------
