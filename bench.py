@@ -6,7 +6,12 @@
     python bench.py --impl reference ...     # times the fp64 CPU oracle on a bounded sample
 
 One step = one pass of the whole path over one packed micro-batch: drk_trloo_advantage over the rollout
-batch, the caller's gather of per-sample advantages, drk_pg_loss_fwd_bwd.  Prints one JSON line.
+batch, drk_segment_advantages (the per-sample advantages of the packed segments), drk_pg_loss_fwd_bwd.
+Prints one JSON line.
+
+--parallelism vocab (not the default) splits W by rows over the ranks instead of giving every rank its own
+micro-batch: drk_pg_shard_stats_fwd, all-gather of the per-row statistics, drk_pg_shard_loss_bwd, all-reduce
+of dH; the same micro-batch on every rank, so the scaling is strong.
 """
 from __future__ import annotations
 
@@ -224,6 +229,9 @@ def main():
     ap.add_argument("--engine", default="auto", choices=["auto", "1cta"],
                     help="auto: tcgen05 kernels on CTA pairs; 1cta: one CTA per tile")
     ap.add_argument("--mrs", default="wide", choices=["wide", "paper", "off"])
+    ap.add_argument("--parallelism", default="data", choices=["data", "vocab"],
+                    help="data: one micro-batch per rank, no collective on the loss path (weak scaling); "
+                         "vocab: W split by rows over the ranks, one micro-batch for all (strong scaling)")
     ap.add_argument("--ref-tokens", type=int, default=256)
     ap.add_argument("--cpu-tokens", type=int, default=512)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -254,9 +262,19 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     B.load()
 
-    # every rank owns a different micro-batch of the same rollout batch (weak scaling)
-    wl = workload.build(args.workload, dev, seed=2000, microbatch=rank, T_override=args.tokens or None)
-    T, H, V, S = wl.T, wl.H, wl.V, wl.S
+    # data parallel: every rank owns a different micro-batch of the same rollout batch (weak scaling);
+    # vocabulary parallel: every rank sees the same micro-batch and owns a block of W's rows (strong scaling)
+    vocab = args.parallelism == "vocab"
+    wl = workload.build(args.workload, dev, seed=2000, microbatch=0 if vocab else rank,
+                        T_override=args.tokens or None)
+    T, H, V_total, S = wl.T, wl.H, wl.V, wl.S
+    v_begin, v_end = dp.vocab_shards(V_total, world)[rank] if vocab else (0, V_total)
+    if v_end <= v_begin:
+        raise SystemExit("more ranks than vocabulary tiles")
+    W_local = wl.W[v_begin:v_end].contiguous() if vocab else wl.W
+    if vocab:
+        wl.W = None
+    V = v_end - v_begin
     code = B.DRK_F32 if wl.dtype == torch.float32 else B.DRK_BF16
     p = B.drk_pg_params_default()
     if args.mrs == "wide":
@@ -273,10 +291,15 @@ def main():
     ret = torch.empty_like(wl.reward)
     adv = torch.empty_like(wl.reward)
     gsize = torch.empty((R, Tmax), dtype=torch.int32, device=dev)
-    seg_flat = (wl.seg_rollout * Tmax + wl.seg_turn).contiguous()
+    seg_rollout = wl.seg_rollout.to(torch.int32).contiguous()
+    seg_turn = wl.seg_turn.to(torch.int32).contiguous()
+    seg_adv = torch.empty(S, dtype=torch.float32, device=dev)
+    stats = torch.empty((T, 4), dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()
     launches = [0]
     comm = None
+    if args.sync_dw and vocab:
+        raise SystemExit("--sync-dw belongs to data parallelism: with W split by rows every rank owns its rows of dW")
     if args.sync_dw:
         # one event per vocabulary chunk; the communication stream reduces a slice of dW once its event fired
         n_chunks, vc = B.drk_pg_bwd_chunks(T, H, V, code, p)
@@ -291,8 +314,13 @@ def main():
         B.drk_trloo_advantage(wl.reward, wl.valid, wl.prompt_of_rollout, R, Tmax, 1.0, B.DRK_BASELINE_TRLOO,
                               ret, adv, gsize, stream)
         launches[0] += B.drk_last_launch_count()
-        seg_adv = adv.view(-1).index_select(0, seg_flat)     # the caller's gather of per-sample advantages
-        B.drk_pg_loss_fwd_bwd(hidden, wl.W, code, ids, rl, mask, cu, seg_adv, T, H, V, S, p, o.loss, o.logp,
+        B.drk_segment_advantages(adv, seg_rollout, seg_turn, R, Tmax, S, seg_adv, o.status, stream)
+        launches[0] += B.drk_last_launch_count()
+        if vocab:
+            launches[0] += dp.vocab_parallel_loss_fwd_bwd(hidden, W_local, ids, rl, mask, cu, seg_adv, v_begin, V_total,
+                                                          p, o, stats, stream)
+            return
+        B.drk_pg_loss_fwd_bwd(hidden, W_local, code, ids, rl, mask, cu, seg_adv, T, H, V, S, p, o.loss, o.logp,
                               o.lse, o.entropy, o.seg_w, o.seg_keep, o.counters, o.dH, o.dW,
                               o.workspace, o.workspace_bytes, o.status, stream)
         launches[0] += B.drk_last_launch_count()
@@ -326,19 +354,26 @@ def main():
     status = int(bufs.status.item())
     counters = bufs.counters.tolist()
     ms_max = dp.max_over_ranks(ms, dev)
-    value = world * T * args.steps / (ms_max * 1e-3)
+    value = (1 if vocab else world) * T * args.steps / (ms_max * 1e-3)
 
     # ---------------------------------------------------------------- the fused call alone (roofline)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    seg_adv = adv.view(-1).index_select(0, seg_flat)
+    fused_launches = [0]
 
     def time_fused(pp, reps):
         out = []
         for _ in range(reps):
             e0.record(stream)
-            B.drk_pg_loss_fwd_bwd(wl.hidden, wl.W, code, wl.ids, wl.rollout_logp, wl.loss_mask, wl.cu, seg_adv, T, H,
-                                  V, S, pp, bufs.loss, bufs.logp, bufs.lse, bufs.entropy, bufs.seg_w, bufs.seg_keep, bufs.counters,
-                                  bufs.dH, bufs.dW, bufs.workspace, bufs.workspace_bytes, bufs.status, stream)
+            if vocab:      # this rank's two calls with the exchange between them
+                fused_launches[0] = dp.vocab_parallel_loss_fwd_bwd(wl.hidden, W_local, wl.ids, wl.rollout_logp,
+                                                                   wl.loss_mask, wl.cu, seg_adv, v_begin, V_total, pp,
+                                                                   bufs, stats, stream)
+            else:
+                B.drk_pg_loss_fwd_bwd(wl.hidden, W_local, code, wl.ids, wl.rollout_logp, wl.loss_mask, wl.cu, seg_adv,
+                                      T, H, V, S, pp, bufs.loss, bufs.logp, bufs.lse, bufs.entropy, bufs.seg_w,
+                                      bufs.seg_keep, bufs.counters, bufs.dH, bufs.dW, bufs.workspace,
+                                      bufs.workspace_bytes, bufs.status, stream)
+                fused_launches[0] = B.drk_last_launch_count()
             e1.record(stream)
             torch.cuda.synchronize()
             out.append(e0.elapsed_time(e1))
@@ -353,8 +388,9 @@ def main():
         return int((per_seg * keep.long()).sum().item())
 
     fused_ms = time_fused(p, min(args.steps, 5))
-    # merge + 3 MRS + 4 compaction kernels are not GEMM launches (the FFMA path has no compaction)
-    n_gemm_launches = B.drk_last_launch_count() - (8 if code == B.DRK_BF16 else 4)
+    # merge + 3 MRS + 4 compaction kernels are not GEMM launches (the FFMA path has no compaction; the
+    # vocabulary-parallel form has one more merge)
+    n_gemm_launches = fused_launches[0] - (8 if code == B.DRK_BF16 else 4) - (1 if vocab else 0)
     Tc = backward_rows() if code == B.DRK_BF16 else T
     Tf = int(bufs.counters[1].item()) if (p.forward_rows == 1 and code == B.DRK_BF16) else T   # rows the forward ran on
     flops = (2.0 * Tf + 6.0 * Tc) * H * V
@@ -363,8 +399,8 @@ def main():
     # DRAM bytes (read + write) of one fused call, from a one-pass ncu capture of exactly this configuration
     # with the kernels as they are; unknown (null) for any other configuration.
     traffic = None
-    if (args.workload, T, args.mrs, args.dw_dtype, args.dh_dtype, args.v_chunk, args.engine, args.forward_rows) == \
-            ("qwen3-14b", 32768, "wide", "f32", "bf16", 0, "auto", "all"):
+    if (args.workload, T, args.mrs, args.dw_dtype, args.dh_dtype, args.v_chunk, args.engine, args.forward_rows,
+            args.parallelism) == ("qwen3-14b", 32768, "wide", "f32", "bf16", 0, "auto", "all", "data"):
         traffic = 165.37e9
     # the same call with rejection switched off: every loss-masked token goes through the backward
     p_off = B.drk_pg_params_default()
@@ -442,7 +478,7 @@ def main():
         ev1.record(stream)
         barrier()
         e_ms = dp.max_over_ranks(ev0.elapsed_time(ev1), dev)
-        e2e = {"value": world * T * args.steps / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e = {"value": (1 if vocab else world) * T * args.steps / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": e_ms / args.steps,
                "what": "every step: hidden, ids, rollout log-probs, mask, cu_seqlens copied from pinned host memory; "
                        "loss, counters, log-probs, keep flags and dH copied back to pinned host memory; uploads and "
@@ -456,16 +492,19 @@ def main():
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True,
+            "scaling": "strong" if vocab else "weak",
             "vs_baseline": None, "dtype": "bf16" if code == B.DRK_BF16 else "f32", "data": "synthetic",
-            "config": {"workload": f"{wl.name}-shaped packed micro-batch", "T": T, "H": H, "V": V, "segments": S,
+            "config": {"workload": f"{wl.name}-shaped packed micro-batch", "T": T, "H": H, "V": V_total, "V_local": V, "segments": S,
                        "rollout_batch": f"{R} rollouts x {Tmax} turns", "mrs": args.mrs,
                        "dW": args.dw_dtype, "dH": args.dh_dtype, "v_chunk": args.v_chunk or "default",
                        "engine": args.engine, "forward_rows": args.forward_rows,
                        "l2": "inputs exceed L2 (W alone is %.2f GB); no flush" % (V * H * 2 / 1e9),
-                       "parallelism": f"dp{world}: one micro-batch per rank, " +
-                                      ("dW all-reduced per vocabulary chunk, overlapped" if args.sync_dw
-                                       else "no collective on the loss path")},
+                       "parallelism": (f"vp{world}: W split by rows ({V} of {V_total} on rank 0), one micro-batch for "
+                                       "all ranks; all-gather of per-row statistics, all-reduce of dH") if vocab else
+                                      (f"dp{world}: one micro-batch per rank, " +
+                                       ("dW all-reduced per vocabulary chunk, overlapped" if args.sync_dw
+                                        else "no collective on the loss path"))},
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s",
                          "frac": achieved / peaks["tflops"], "traffic": traffic,
                          "kernel": "umma_gemm_kernel (all four instantiations inside one drk_pg_loss_fwd_bwd call)",

@@ -82,6 +82,17 @@ int drk_trloo_advantage(const float* reward, const uint8_t* valid,
                         int32_t* gsize, void* stream);
 
 /*
+ * Per-sample advantages of a packed micro-batch.  Every turn of a trajectory is one training sample
+ * (Sec. 4.3); segment g holds turn seg_turn[g] of rollout seg_rollout[g] and takes
+ *   seg_adv[g] = adv[seg_rollout[g] * Tmax + seg_turn[g]]
+ * from the table drk_trloo_advantage wrote.  adv [R*Tmax] float, seg_rollout, seg_turn [S] int32, seg_adv [S]
+ * float, status [1] uint32: device.  An index outside the table gives seg_adv[g] = 0 and sets
+ * DRK_STATUS_BAD_SEGMENTS.  S = 0 enqueues nothing.
+ */
+int drk_segment_advantages(const float* adv, const int32_t* seg_rollout, const int32_t* seg_turn, int32_t R,
+                           int32_t Tmax, int32_t S, float* seg_adv, uint32_t* status, void* stream);
+
+/*
  * Reward front-end, upstream of drk_trloo_advantage: per-sample reward and the retention decision of
  * profiling-based rejection sampling.
  *
@@ -245,6 +256,46 @@ int drk_pg_loss_fwd_bwd(const void* hidden, const void* W, int32_t in_dtype, con
                         float* lse, float* entropy, float* seg_w, uint8_t* seg_keep, int64_t* counters,
                         void* dH, void* dW, void* workspace, size_t workspace_bytes, uint32_t* status,
                         void* stream);
+
+/*
+ * The same path when the LM head is split by vocabulary rows over several GPUs (each holding rows
+ * [v_begin, v_begin + V_local) of W: W_shard is that block, [V_local, H] row-major).  The paper does not
+ * say how its trainer lays out the LM head; these two calls compute exactly the quantities defined above
+ * (Sec. 5.1 log-probs and rejection, App. A loss and gradient), arranged so that every rank touches only its
+ * own rows of W and the ranks exchange two small tensors.  The exchanges are the caller's (this library makes
+ * no collective call):
+ *
+ *   1. every rank:  drk_pg_shard_stats_fwd  ->  stats [T,4] float, per row t over the rank's columns
+ *          m = max_v s[t,v]     l = sum_v exp(s[t,v] - m)     r = sum_v exp(s[t,v] - m) * s[t,v]
+ *          g = s[t, ids[t]] if v_begin <= ids[t] < v_begin + V_local, else 0
+ *   2. all-gather of stats over the ranks  ->  stats_all [n_shards, T, 4] (any order of the ranks)
+ *   3. every rank:  drk_pg_shard_loss_bwd   (same arguments as drk_pg_loss_fwd_bwd, plus stats_all)
+ *          M = max_k m_k   L = sum_k l_k exp(m_k - M)   lse = M + log L   logp = sum_k g_k - lse
+ *          entropy = lse - (sum_k r_k exp(m_k - M)) / L
+ *          then rejection sampling, coefficients and loss as in drk_pg_loss_fwd_bwd: loss, logp, lse,
+ *          entropy, seg_w, seg_keep and counters come out identical on every rank;
+ *          dW_shard [V_local, H] = rows v_begin.. of dW, final;
+ *          dH_part [T, H] = sum over the rank's columns of dL[t,v] W[v,:]
+ *   4. all-reduce (sum) of dH_part over the ranks = dH.  p->dh_dtype = DRK_F32 keeps that sum in fp32.
+ *
+ * ids hold token numbers of the whole vocabulary, 0 <= ids[t] < V_total; ids outside set DRK_STATUS_BAD_ID in
+ * step 3.  Workspace: drk_pg_workspace_bytes(T, H, V_local, S, in_dtype, p, which) with which = 0 for step 1
+ * and 1 for step 3.  p->forward_rows must be 0 in step 3 (DRK_ERR_UNSUPPORTED otherwise).  n_shards <= 4096.
+ * stats and stats_all must be 16-byte aligned.  Every other argument, limit, status bit and return code is that
+ * of drk_pg_logprob_fwd (step 1) and drk_pg_loss_fwd_bwd (step 3).  With one shard covering the whole
+ * vocabulary the results equal those of drk_pg_loss_fwd_bwd.
+ */
+int drk_pg_shard_stats_fwd(const void* hidden, const void* W_shard, int32_t in_dtype, const int32_t* ids,
+                           int64_t T, int32_t H, int32_t V_local, int32_t v_begin, int32_t V_total,
+                           int32_t engine, float* stats, void* workspace, size_t workspace_bytes,
+                           uint32_t* status, void* stream);
+int drk_pg_shard_loss_bwd(const void* hidden, const void* W_shard, int32_t in_dtype, const int32_t* ids,
+                          const float* stats_all, int32_t n_shards, const float* rollout_logp,
+                          const uint8_t* loss_mask, const int32_t* cu_seqlens, const float* seg_adv,
+                          int64_t T, int32_t H, int32_t V_local, int32_t v_begin, int32_t V_total, int32_t S,
+                          const drk_pg_params* p, float* loss, float* logp, float* lse, float* entropy,
+                          float* seg_w, uint8_t* seg_keep, int64_t* counters, void* dH_part, void* dW_shard,
+                          void* workspace, size_t workspace_bytes, uint32_t* status, void* stream);
 
 /*
  * Stability diagnostics of one micro-batch, from the outputs of the calls above: what the paper

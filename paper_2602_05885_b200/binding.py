@@ -120,6 +120,14 @@ def load() -> ctypes.CDLL:
     lib.drk_pg_diagnostics.argtypes = [vp, vp, vp, vp, vp, i64, i32, vp, i32, vp, i32, i32, i32, vp, vp]
     lib.drk_pg_diagnostics.restype = ctypes.c_int
     lib.drk_pg_loss_fwd_bwd.restype = ctypes.c_int
+    lib.drk_pg_shard_stats_fwd.argtypes = [vp, vp, i32, vp, i64, i32, i32, i32, i32, i32, vp, vp, sz, vp, vp]
+    lib.drk_pg_shard_stats_fwd.restype = ctypes.c_int
+    lib.drk_pg_shard_loss_bwd.argtypes = [vp, vp, i32, vp, vp, i32, vp, vp, vp, vp, i64, i32, i32, i32, i32, i32,
+                                          ctypes.POINTER(drk_pg_params), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz,
+                                          vp, vp]
+    lib.drk_pg_shard_loss_bwd.restype = ctypes.c_int
+    lib.drk_segment_advantages.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp]
+    lib.drk_segment_advantages.restype = ctypes.c_int
     lib.drk_last_launch_count.argtypes = []
     lib.drk_last_launch_count.restype = ctypes.c_int
     lib.drk_status_string.argtypes = [ctypes.c_int]
@@ -255,6 +263,41 @@ def drk_pg_loss_fwd_bwd(hidden, W, in_dtype: int, ids, rollout_logp, loss_mask, 
                                     _ptr(workspace), workspace_bytes, _ptr(status), _stream(stream))
     if check and rc != DRK_OK:
         raise DrkError(rc, "drk_pg_loss_fwd_bwd")
+    return rc
+
+
+def drk_pg_shard_stats_fwd(hidden, W_shard, in_dtype: int, ids, T: int, H: int, V_local: int, v_begin: int,
+                           V_total: int, engine: int, stats, workspace, workspace_bytes: int, status, stream=None,
+                           check: bool = True) -> int:
+    rc = load().drk_pg_shard_stats_fwd(_ptr(hidden), _ptr(W_shard), in_dtype, _ptr(ids), T, H, V_local, v_begin,
+                                       V_total, engine, _ptr(stats), _ptr(workspace), workspace_bytes, _ptr(status),
+                                       _stream(stream))
+    if check and rc != DRK_OK:
+        raise DrkError(rc, "drk_pg_shard_stats_fwd")
+    return rc
+
+
+def drk_pg_shard_loss_bwd(hidden, W_shard, in_dtype: int, ids, stats_all, n_shards: int, rollout_logp, loss_mask,
+                          cu_seqlens, seg_adv, T: int, H: int, V_local: int, v_begin: int, V_total: int, S: int,
+                          p: Optional[drk_pg_params], loss, logp, lse, entropy, seg_w, seg_keep, counters, dH_part,
+                          dW_shard, workspace, workspace_bytes: int, status, stream=None, check: bool = True) -> int:
+    rc = load().drk_pg_shard_loss_bwd(_ptr(hidden), _ptr(W_shard), in_dtype, _ptr(ids), _ptr(stats_all), n_shards,
+                                      _ptr(rollout_logp), _ptr(loss_mask), _ptr(cu_seqlens), _ptr(seg_adv), T, H,
+                                      V_local, v_begin, V_total, S, ctypes.byref(p) if p is not None else None,
+                                      _ptr(loss), _ptr(logp), _ptr(lse), _ptr(entropy), _ptr(seg_w), _ptr(seg_keep),
+                                      _ptr(counters), _ptr(dH_part), _ptr(dW_shard), _ptr(workspace), workspace_bytes,
+                                      _ptr(status), _stream(stream))
+    if check and rc != DRK_OK:
+        raise DrkError(rc, "drk_pg_shard_loss_bwd")
+    return rc
+
+
+def drk_segment_advantages(adv, seg_rollout, seg_turn, R: int, Tmax: int, S: int, seg_adv, status, stream=None,
+                           check: bool = True) -> int:
+    rc = load().drk_segment_advantages(_ptr(adv), _ptr(seg_rollout), _ptr(seg_turn), R, Tmax, S, _ptr(seg_adv),
+                                       _ptr(status), _stream(stream))
+    if check and rc != DRK_OK:
+        raise DrkError(rc, "drk_segment_advantages")
     return rc
 
 

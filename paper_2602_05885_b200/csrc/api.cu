@@ -140,14 +140,130 @@ bool params_ok(const drk_pg_params& p) {
 int run_fwd(const void* hidden, const void* W, int in_dtype, const int32_t* ids, int64_t T, int H, int V,
             bool simt, int engine, const FwdWs& w, float* logp, float* lse, float* entropy, uint32_t* status,
             cudaStream_t st, const __nv_bfloat16* hidden_c = nullptr, const int32_t* rowmap = nullptr,
-            const int32_t* n_rows = nullptr) {
+            const int32_t* n_rows = nullptr, int id_off = 0, float* stats = nullptr) {
   if (simt) {
     SimtFwdArgs a{hidden, W, in_dtype, ids, T, H, V, logp, lse, w.part, w.tgt, w.nsplit, status, entropy};
+    a.id_off = id_off; a.stats = stats;
     return launch_simt_fwd(a, st);
   }
   UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, w.part, w.tgt, w.nsplit, status, umma_ctas(engine), entropy,
                 hidden_c, rowmap, n_rows};
+  a.id_off = id_off; a.stats = stats;
   return launch_umma_fwd(a, st);
+}
+
+// Vocabulary-range mode of the fused call: log-probs come from all ranges' statistics instead of a forward
+// pass, and W holds columns [v_begin, v_begin + V) of a vocabulary of V_total columns.
+struct ShardCtx {
+  const float* stats_all; int n_shards; int v_begin; int V_total;
+};
+
+bool shard_ok(int V_local, int v_begin, int V_total) {
+  return V_local >= 1 && v_begin >= 0 && V_total >= 1 && V_total <= (1 << 24) &&
+         (int64_t)v_begin + V_local <= V_total;
+}
+
+int loss_fwd_bwd_impl(const void* hidden, const void* W, int32_t in_dtype, const int32_t* ids,
+                      const float* rollout_logp, const uint8_t* loss_mask, const int32_t* cu_seqlens,
+                      const float* seg_adv, int64_t T, int32_t H, int32_t V, int32_t S, const drk_pg_params* pp,
+                      float* loss, float* logp, float* lse, float* entropy, float* seg_w, uint8_t* seg_keep,
+                      int64_t* counters, void* dH, void* dW, void* workspace, size_t workspace_bytes, uint32_t* status,
+                      void* stream, const ShardCtx* sh) {
+  g_launches = 0;
+  drk_pg_params p;
+  if (pp) p = *pp; else drk_pg_params_default(&p);
+  if (!sizes_ok(T, H, V, in_dtype) || S < 0 || S > (1 << 24) || !params_ok(p)) return DRK_ERR_INVALID_ARG;
+  if (!W || !dW || !loss || !counters || !workspace || !status) return DRK_ERR_INVALID_ARG;
+  if (T > 0 && (!hidden || !ids || !rollout_logp || !loss_mask || !logp || !lse || !dH)) return DRK_ERR_INVALID_ARG;
+  if (S > 0 && (!cu_seqlens || !seg_adv || !seg_w || !seg_keep)) return DRK_ERR_INVALID_ARG;
+  if (!aligned(hidden, 16) || !aligned(W, 16) || !aligned(dH, 16) || !aligned(dW, 16) || !aligned(workspace, 256) ||
+      !aligned(logp, 16) || !aligned(rollout_logp, 16) || !aligned(loss_mask, 4))
+    return DRK_ERR_INVALID_ARG;
+  if (sh != nullptr) {
+    if (!shard_ok(V, sh->v_begin, sh->V_total) || sh->n_shards < 1 || sh->n_shards > 4096) return DRK_ERR_INVALID_ARG;
+    if (T > 0 && (!sh->stats_all || !aligned(sh->stats_all, 16))) return DRK_ERR_INVALID_ARG;
+    if (p.forward_rows != 0) return DRK_ERR_UNSUPPORTED;   // there is no forward pass to restrict
+  }
+  const bool simt = use_simt(in_dtype, p.engine);
+  if (!simt && (H % 8) != 0) return DRK_ERR_UNSUPPORTED;
+  if (workspace_bytes < drk_pg_workspace_bytes(T, H, V, S, in_dtype, &p, 1)) return DRK_ERR_WORKSPACE;
+  if (p.dw_chunk_events != nullptr) {
+    const int vc = round_vchunk(p.v_chunk, T, H, V, simt);
+    if (T == 0 || p.n_dw_chunk_events != (int)ceil_div(V, vc)) return DRK_ERR_INVALID_ARG;
+    for (int i = 0; i < p.n_dw_chunk_events; ++i)
+      if (p.dw_chunk_events[i] == nullptr) return DRK_ERR_INVALID_ARG;
+  }
+  int rc = check_arch();
+  if (rc != DRK_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  Carver c(workspace);
+  const FwdWs fw = carve_fwd(c, T, V, simt, p.engine);
+  const BwdWs bw = carve_bwd(c, T, H, V, S, simt, p);
+  const int id_off = sh ? sh->v_begin : 0;
+
+  auto fail = [&](int code) { g_launches = 0; return code; };
+
+  if (T > 0 && sh != nullptr) {
+    rc = launch_shard_merge(sh->stats_all, sh->n_shards, ids, T, sh->V_total, logp, lse, entropy, status, st);
+    if (rc != DRK_OK) return fail(rc);
+  } else if (T > 0 && p.forward_rows == 1 && !simt) {
+    // forward over the rows the loss can use: loss-masked tokens inside segments; the rest read 0
+    rc = launch_need_rows(loss_mask, cu_seqlens, T, S, bw.coeff, st);
+    if (rc != DRK_OK) return fail(rc);
+    CompactArgs ca{bw.coeff, static_cast<const __nv_bfloat16*>(hidden), T, H, bw.blk_cnt, bw.blk_off, bw.n_rows,
+                   bw.rowmap, bw.hidden_c};
+    rc = launch_compact(ca, st);
+    if (rc != DRK_OK) return fail(rc);
+    if (cudaMemsetAsync(logp, 0, sizeof(float) * (size_t)T, st) != cudaSuccess ||
+        cudaMemsetAsync(lse, 0, sizeof(float) * (size_t)T, st) != cudaSuccess ||
+        (entropy && cudaMemsetAsync(entropy, 0, sizeof(float) * (size_t)T, st) != cudaSuccess))
+      return fail(DRK_ERR_CUDA);
+    rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, p.engine, fw, logp, lse, entropy, status, st, bw.hidden_c,
+                 bw.rowmap, bw.n_rows);
+    if (rc != DRK_OK) return fail(rc);
+  } else if (T > 0) {
+    rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, p.engine, fw, logp, lse, entropy, status, st);
+    if (rc != DRK_OK) return fail(rc);
+  }
+  MrsArgs m{};
+  m.logp = logp; m.rollout_logp = rollout_logp; m.loss_mask = loss_mask; m.cu = cu_seqlens; m.seg_adv = seg_adv;
+  m.T = T; m.S = S;
+  m.ln_lo = p.mrs_lo > 0.f ? std::log((double)p.mrs_lo) : -std::numeric_limits<double>::infinity();
+  m.ln_hi = std::isinf(p.mrs_hi) ? std::numeric_limits<double>::infinity() : std::log((double)p.mrs_hi);
+  m.ln_veto = p.veto_ratio > 0.f ? std::log((double)p.veto_ratio) : -std::numeric_limits<double>::infinity();
+  m.norm = p.norm; m.explicit_scale = p.explicit_scale; m.keep_from_caller = p.keep_from_caller;
+  m.seg_w = seg_w; m.seg_keep = seg_keep; m.loss = loss; m.counters = counters; m.coeff = bw.coeff;
+  m.seg_stats = bw.seg_stats; m.status = status;
+  rc = launch_mrs(m, st);
+  if (rc != DRK_OK) return fail(rc);
+
+  if (T == 0) {
+    // no tokens: gradients are zero
+    if (!p.dw_accumulate) {
+      const size_t esz = p.dw_dtype == DRK_BF16 ? 2 : 4;
+      if (cudaMemsetAsync(dW, 0, esz * (size_t)V * (size_t)H, st) != cudaSuccess) return fail(DRK_ERR_CUDA);
+    }
+    return DRK_OK;
+  }
+  if (simt) {
+    SimtBwdArgs b{hidden, W, in_dtype, ids, T, H, V, lse, bw.coeff, static_cast<float*>(bw.dL), bw.vc,
+                  dH, p.dh_dtype, bw.dH_acc, dW, p.dw_dtype, p.dw_accumulate, p.dw_chunk_events};
+    b.id_off = id_off;
+    rc = launch_simt_bwd(b, st);
+  } else {
+    CompactArgs ca{bw.coeff, static_cast<const __nv_bfloat16*>(hidden), T, H, bw.blk_cnt, bw.blk_off, bw.n_rows,
+                   bw.rowmap, bw.hidden_c};
+    rc = launch_compact(ca, st);
+    if (rc != DRK_OK) return fail(rc);
+    UmmaBwdArgs b{hidden, W, ids, T, H, V, lse, bw.coeff, static_cast<__nv_bfloat16*>(bw.dL), bw.vc,
+                  dH, p.dh_dtype, bw.dH_acc, dW, p.dw_dtype, p.dw_accumulate, status, umma_ctas(p.engine),
+                  bw.hidden_c, bw.rowmap, bw.n_rows, p.dw_chunk_events};
+    b.id_off = id_off;
+    rc = launch_umma_bwd(b, st);
+  }
+  if (rc != DRK_OK) return fail(rc);
+  return DRK_OK;
 }
 
 }  // namespace
@@ -245,90 +361,62 @@ int drk_pg_loss_fwd_bwd(const void* hidden, const void* W, int32_t in_dtype, con
                         float* loss, float* logp, float* lse, float* entropy, float* seg_w, uint8_t* seg_keep,
                         int64_t* counters, void* dH, void* dW, void* workspace, size_t workspace_bytes, uint32_t* status,
                         void* stream) {
+  return loss_fwd_bwd_impl(hidden, W, in_dtype, ids, rollout_logp, loss_mask, cu_seqlens, seg_adv, T, H, V, S, pp, loss,
+                           logp, lse, entropy, seg_w, seg_keep, counters, dH, dW, workspace, workspace_bytes, status,
+                           stream, nullptr);
+}
+
+int drk_pg_shard_stats_fwd(const void* hidden, const void* W_shard, int32_t in_dtype, const int32_t* ids, int64_t T,
+                           int32_t H, int32_t V_local, int32_t v_begin, int32_t V_total, int32_t engine, float* stats,
+                           void* workspace, size_t workspace_bytes, uint32_t* status, void* stream) {
   g_launches = 0;
-  drk_pg_params p;
-  if (pp) p = *pp; else drk_pg_params_default(&p);
-  if (!sizes_ok(T, H, V, in_dtype) || S < 0 || S > (1 << 24) || !params_ok(p)) return DRK_ERR_INVALID_ARG;
-  if (!W || !dW || !loss || !counters || !workspace || !status) return DRK_ERR_INVALID_ARG;
-  if (T > 0 && (!hidden || !ids || !rollout_logp || !loss_mask || !logp || !lse || !dH)) return DRK_ERR_INVALID_ARG;
-  if (S > 0 && (!cu_seqlens || !seg_adv || !seg_w || !seg_keep)) return DRK_ERR_INVALID_ARG;
-  if (!aligned(hidden, 16) || !aligned(W, 16) || !aligned(dH, 16) || !aligned(dW, 16) || !aligned(workspace, 256) ||
-      !aligned(logp, 16) || !aligned(rollout_logp, 16) || !aligned(loss_mask, 4))
+  if (!sizes_ok(T, H, V_local, in_dtype) || !shard_ok(V_local, v_begin, V_total)) return DRK_ERR_INVALID_ARG;
+  if (!engine_ok(engine)) return DRK_ERR_INVALID_ARG;
+  if (T == 0) return DRK_OK;
+  if (!hidden || !W_shard || !ids || !stats || !workspace || !status) return DRK_ERR_INVALID_ARG;
+  if (!aligned(hidden, 16) || !aligned(W_shard, 16) || !aligned(stats, 16) || !aligned(workspace, 256))
     return DRK_ERR_INVALID_ARG;
-  const bool simt = use_simt(in_dtype, p.engine);
+  const bool simt = use_simt(in_dtype, engine);
   if (!simt && (H % 8) != 0) return DRK_ERR_UNSUPPORTED;
-  if (workspace_bytes < drk_pg_workspace_bytes(T, H, V, S, in_dtype, &p, 1)) return DRK_ERR_WORKSPACE;
-  if (p.dw_chunk_events != nullptr) {
-    const int vc = round_vchunk(p.v_chunk, T, H, V, simt);
-    if (T == 0 || p.n_dw_chunk_events != (int)ceil_div(V, vc)) return DRK_ERR_INVALID_ARG;
-    for (int i = 0; i < p.n_dw_chunk_events; ++i)
-      if (p.dw_chunk_events[i] == nullptr) return DRK_ERR_INVALID_ARG;
-  }
+  drk_pg_params p;
+  drk_pg_params_default(&p);
+  p.engine = engine;
+  if (workspace_bytes < drk_pg_workspace_bytes(T, H, V_local, 0, in_dtype, &p, 0)) return DRK_ERR_WORKSPACE;
   int rc = check_arch();
   if (rc != DRK_OK) return rc;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-
   Carver c(workspace);
-  const FwdWs fw = carve_fwd(c, T, V, simt, p.engine);
-  const BwdWs bw = carve_bwd(c, T, H, V, S, simt, p);
+  const FwdWs w = carve_fwd(c, T, V_local, simt, engine);
+  rc = run_fwd(hidden, W_shard, in_dtype, ids, T, H, V_local, simt, engine, w, nullptr, nullptr, nullptr, status,
+               static_cast<cudaStream_t>(stream), nullptr, nullptr, nullptr, v_begin, stats);
+  if (rc != DRK_OK) g_launches = 0;
+  return rc;
+}
 
-  auto fail = [&](int code) { g_launches = 0; return code; };
+int drk_pg_shard_loss_bwd(const void* hidden, const void* W_shard, int32_t in_dtype, const int32_t* ids,
+                          const float* stats_all, int32_t n_shards, const float* rollout_logp,
+                          const uint8_t* loss_mask, const int32_t* cu_seqlens, const float* seg_adv, int64_t T,
+                          int32_t H, int32_t V_local, int32_t v_begin, int32_t V_total, int32_t S,
+                          const drk_pg_params* p, float* loss, float* logp, float* lse, float* entropy, float* seg_w,
+                          uint8_t* seg_keep, int64_t* counters, void* dH_part, void* dW_shard, void* workspace,
+                          size_t workspace_bytes, uint32_t* status, void* stream) {
+  const ShardCtx sh{stats_all, n_shards, v_begin, V_total};
+  return loss_fwd_bwd_impl(hidden, W_shard, in_dtype, ids, rollout_logp, loss_mask, cu_seqlens, seg_adv, T, H, V_local,
+                           S, p, loss, logp, lse, entropy, seg_w, seg_keep, counters, dH_part, dW_shard, workspace,
+                           workspace_bytes, status, stream, &sh);
+}
 
-  if (T > 0 && p.forward_rows == 1 && !simt) {
-    // forward over the rows the loss can use: loss-masked tokens inside segments; the rest read 0
-    rc = launch_need_rows(loss_mask, cu_seqlens, T, S, bw.coeff, st);
-    if (rc != DRK_OK) return fail(rc);
-    CompactArgs ca{bw.coeff, static_cast<const __nv_bfloat16*>(hidden), T, H, bw.blk_cnt, bw.blk_off, bw.n_rows,
-                   bw.rowmap, bw.hidden_c};
-    rc = launch_compact(ca, st);
-    if (rc != DRK_OK) return fail(rc);
-    if (cudaMemsetAsync(logp, 0, sizeof(float) * (size_t)T, st) != cudaSuccess ||
-        cudaMemsetAsync(lse, 0, sizeof(float) * (size_t)T, st) != cudaSuccess ||
-        (entropy && cudaMemsetAsync(entropy, 0, sizeof(float) * (size_t)T, st) != cudaSuccess))
-      return fail(DRK_ERR_CUDA);
-    rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, p.engine, fw, logp, lse, entropy, status, st, bw.hidden_c,
-                 bw.rowmap, bw.n_rows);
-    if (rc != DRK_OK) return fail(rc);
-  } else if (T > 0) {
-    rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, p.engine, fw, logp, lse, entropy, status, st);
-    if (rc != DRK_OK) return fail(rc);
-  }
-  MrsArgs m{};
-  m.logp = logp; m.rollout_logp = rollout_logp; m.loss_mask = loss_mask; m.cu = cu_seqlens; m.seg_adv = seg_adv;
-  m.T = T; m.S = S;
-  m.ln_lo = p.mrs_lo > 0.f ? std::log((double)p.mrs_lo) : -std::numeric_limits<double>::infinity();
-  m.ln_hi = std::isinf(p.mrs_hi) ? std::numeric_limits<double>::infinity() : std::log((double)p.mrs_hi);
-  m.ln_veto = p.veto_ratio > 0.f ? std::log((double)p.veto_ratio) : -std::numeric_limits<double>::infinity();
-  m.norm = p.norm; m.explicit_scale = p.explicit_scale; m.keep_from_caller = p.keep_from_caller;
-  m.seg_w = seg_w; m.seg_keep = seg_keep; m.loss = loss; m.counters = counters; m.coeff = bw.coeff;
-  m.seg_stats = bw.seg_stats; m.status = status;
-  rc = launch_mrs(m, st);
-  if (rc != DRK_OK) return fail(rc);
-
-  if (T == 0) {
-    // no tokens: gradients are zero
-    if (!p.dw_accumulate) {
-      const size_t esz = p.dw_dtype == DRK_BF16 ? 2 : 4;
-      if (cudaMemsetAsync(dW, 0, esz * (size_t)V * (size_t)H, st) != cudaSuccess) return fail(DRK_ERR_CUDA);
-    }
-    return DRK_OK;
-  }
-  if (simt) {
-    SimtBwdArgs b{hidden, W, in_dtype, ids, T, H, V, lse, bw.coeff, static_cast<float*>(bw.dL), bw.vc,
-                  dH, p.dh_dtype, bw.dH_acc, dW, p.dw_dtype, p.dw_accumulate, p.dw_chunk_events};
-    rc = launch_simt_bwd(b, st);
-  } else {
-    CompactArgs ca{bw.coeff, static_cast<const __nv_bfloat16*>(hidden), T, H, bw.blk_cnt, bw.blk_off, bw.n_rows,
-                   bw.rowmap, bw.hidden_c};
-    rc = launch_compact(ca, st);
-    if (rc != DRK_OK) return fail(rc);
-    UmmaBwdArgs b{hidden, W, ids, T, H, V, lse, bw.coeff, static_cast<__nv_bfloat16*>(bw.dL), bw.vc,
-                  dH, p.dh_dtype, bw.dH_acc, dW, p.dw_dtype, p.dw_accumulate, status, umma_ctas(p.engine),
-                  bw.hidden_c, bw.rowmap, bw.n_rows, p.dw_chunk_events};
-    rc = launch_umma_bwd(b, st);
-  }
-  if (rc != DRK_OK) return fail(rc);
-  return DRK_OK;
+int drk_segment_advantages(const float* adv, const int32_t* seg_rollout, const int32_t* seg_turn, int32_t R,
+                           int32_t Tmax, int32_t S, float* seg_adv, uint32_t* status, void* stream) {
+  g_launches = 0;
+  if (R < 0 || Tmax < 0 || S < 0) return DRK_ERR_INVALID_ARG;
+  if (S == 0) return DRK_OK;
+  if (!seg_rollout || !seg_turn || !seg_adv || !status || (!adv && (int64_t)R * Tmax > 0)) return DRK_ERR_INVALID_ARG;
+  int rc = check_arch();
+  if (rc != DRK_OK) return rc;
+  rc = launch_segment_advantages(adv, seg_rollout, seg_turn, R, Tmax, S, seg_adv, status,
+                                 static_cast<cudaStream_t>(stream));
+  if (rc != DRK_OK) g_launches = 0;
+  return rc;
 }
 
 int drk_last_launch_count(void) { return g_launches; }

@@ -31,6 +31,13 @@ template <typename T> __device__ __forceinline__ float to_f32(T x);
 template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
 template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
 
+// Token id relative to the vocabulary range [id_off, id_off + width): the local column, or -1 when the
+// token belongs to another range (or is invalid).
+__device__ __forceinline__ int local_id(int id, int id_off, int width) {
+  const uint32_t rel = (uint32_t)id - (uint32_t)id_off;
+  return rel < (uint32_t)width ? (int)rel : -1;
+}
+
 // ---- internal launchers (each returns a drk_status) -------------------------------------------
 
 int launch_trloo(const float* reward, const uint8_t* valid, const int32_t* prompt, int R, int Tmax,
@@ -45,24 +52,37 @@ struct MrsArgs {
   double* seg_stats /*[S*4] workspace*/; uint32_t* status;
 };
 int launch_mrs(const MrsArgs& a, cudaStream_t st);
+// seg_adv[g] = adv[seg_rollout[g] * Tmax + seg_turn[g]] (0 and a status bit for indices outside the table)
+int launch_segment_advantages(const float* adv, const int32_t* seg_rollout, const int32_t* seg_turn, int R, int Tmax,
+                              int S, float* seg_adv, uint32_t* status, cudaStream_t st);
 
 // FFMA path.
 struct SimtFwdArgs {
   const void* hidden; const void* W; int in_dtype; const int32_t* ids; int64_t T; int H; int V;
   float* logp; float* lse; float* part /*[nsplit*T*4]*/; float* tgt /*[T]*/; int nsplit; uint32_t* status;
   float* entropy /*[T] or null*/;
+  // vocabulary-range mode: W holds columns [id_off, id_off + V) of a larger vocabulary; when stats is
+  // given the call ends with the range's per-row statistics [T,4] instead of logp / lse
+  int id_off = 0; float* stats = nullptr;
 };
 int simt_nsplit(int64_t T, int V);
 int launch_simt_fwd(const SimtFwdArgs& a, cudaStream_t st);
 int launch_lse_merge(const float* part, const float* tgt, const int32_t* ids, int64_t T, int V, int nsplit,
                      float* logp, float* lse, float* entropy, uint32_t* status, const int32_t* rowmap,
                      const int32_t* n_rows, cudaStream_t st);
+// Vocabulary-range mode: per-row statistics (max, sum-exp, sum-exp-times-logit, target logit or 0) of one
+// range from its partials, and the recombination of all ranges' statistics into logp, lse, entropy.
+int launch_shard_stats(const float* part, const float* tgt, const int32_t* ids, int id_off, int64_t T, int V,
+                       int nsplit, float* stats, uint32_t* status, cudaStream_t st);
+int launch_shard_merge(const float* stats_all, int n_shards, const int32_t* ids, int64_t T, int V_total, float* logp,
+                       float* lse, float* entropy, uint32_t* status, cudaStream_t st);
 struct SimtBwdArgs {
   const void* hidden; const void* W; int in_dtype; const int32_t* ids; int64_t T; int H; int V;
   const float* lse; const float* coeff; float* dL /*[T*vc] fp32 workspace*/; int vc;
   void* dH; int dh_dtype; float* dH_acc /*fp32 [T,H] or null when dH is fp32*/;
   void* dW; int dw_dtype; int dw_accumulate;
   void* const* chunk_events;  // optional cudaEvent_t per vocabulary chunk, recorded when its dW rows are final
+  int id_off = 0;             // W holds columns [id_off, id_off + V) of a larger vocabulary
 };
 int launch_simt_bwd(const SimtBwdArgs& a, cudaStream_t st);
 
@@ -74,6 +94,7 @@ struct UmmaFwdArgs {
   float* entropy /*[T] or null*/;
   // optional: evaluate only the rows listed in rowmap (gathered into hidden_c); others are left untouched
   const __nv_bfloat16* hidden_c; const int32_t* rowmap; const int32_t* n_rows;
+  int id_off = 0; float* stats = nullptr;   // vocabulary-range mode, as in SimtFwdArgs
 };
 int umma_nsplit(int64_t T, int V, int ctas, bool frugal);
 int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st);
@@ -84,6 +105,7 @@ struct UmmaBwdArgs {
   int ctas;
   const __nv_bfloat16* hidden_c; const int32_t* rowmap; const int32_t* n_rows;  // compacted rows
   void* const* chunk_events;  // optional cudaEvent_t per vocabulary chunk, recorded when its dW rows are final
+  int id_off = 0;             // W holds columns [id_off, id_off + V) of a larger vocabulary
 };
 int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st);
 

@@ -65,7 +65,7 @@ template <typename TIn>
 __global__ void __launch_bounds__(kThreads)
 lmhead_fwd_kernel(const TIn* __restrict__ hidden, const TIn* __restrict__ W, const int32_t* __restrict__ ids,
                   int64_t T, int H, int V, int tiles_per_split, float* __restrict__ part,
-                  float* __restrict__ tgt) {
+                  float* __restrict__ tgt, int id_off) {
   // part holds, per vocabulary range and row, {running max m, sum exp(s-m), sum exp(s-m)*s, unused}
   __shared__ __align__(16) float As[BK][BM + 4];
   __shared__ __align__(16) float Bs[BK][BN + 4];
@@ -83,7 +83,7 @@ lmhead_fwd_kernel(const TIn* __restrict__ hidden, const TIn* __restrict__ W, con
     run_l[i] = 0.f;
     run_r[i] = 0.f;
     const int64_t r = row0 + ty * 4 + i;
-    target[i] = (r < T) ? ids[r] : -1;
+    target[i] = (r < T) ? local_id(ids[r], id_off, V) : -1;
   }
   for (int n = n_begin; n < n_end; ++n) {
     const int col0 = n * BN;
@@ -174,7 +174,7 @@ template <typename TIn>
 __global__ void __launch_bounds__(kThreads)
 lmhead_dl_kernel(const TIn* __restrict__ hidden, const TIn* __restrict__ W, const int32_t* __restrict__ ids,
                  const float* __restrict__ lse, const float* __restrict__ coeff, int64_t T, int H, int V,
-                 int v0, int vc_this, int vc, float* __restrict__ dL) {
+                 int v0, int vc_this, int vc, float* __restrict__ dL, int id_off) {
   __shared__ __align__(16) float As[BK][BM + 4];
   __shared__ __align__(16) float Bs[BK][BN + 4];
   const int tid = threadIdx.x, ty = tid / 16, tx = tid % 16;
@@ -187,7 +187,7 @@ lmhead_dl_kernel(const TIn* __restrict__ hidden, const TIn* __restrict__ W, cons
     const int64_t r = row0 + ty * 4 + i;
     if (r >= T) continue;
     const float c = coeff[r], z = lse[r];
-    const int id = ids[r];
+    const int id = local_id(ids[r], id_off, V);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int v = col0 + tx * 4 + j;
@@ -245,6 +245,75 @@ gemm_kernel(const float* __restrict__ A, int64_t a_rs, int64_t a_cs, const TB* _
   }
 }
 
+// Statistics of one vocabulary range per row, from the range's partials: (max, sum-exp, sum-exp-times-logit)
+// relative to that max, and the sampled token's logit if the token lies in the range, else 0.
+__global__ void shard_stats_kernel(const float* __restrict__ part, const float* __restrict__ tgt,
+                                   const int32_t* __restrict__ ids, int id_off, int64_t T, int V, int nsplit,
+                                   float* __restrict__ stats, uint32_t* __restrict__ status) {
+  const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (t >= T) return;
+  const float4* p4 = reinterpret_cast<const float4*>(part);
+  float M = -CUDART_INF_F;
+  for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p4[(int64_t)s * T + t].x);
+  float L = 0.f, R = 0.f;
+  for (int s = 0; s < nsplit; ++s) {
+    const float4 v = p4[(int64_t)s * T + t];
+    if (v.x > -CUDART_INF_F) {
+      const float w = expf(v.x - M);
+      L += v.y * w;
+      R += v.z * w;
+    }
+  }
+  const float tg = local_id(ids[t], id_off, V) >= 0 ? tgt[t] : 0.f;
+  if (!isfinite(M) || !isfinite(L)) atomicOr(status, DRK_STATUS_NONFINITE);
+  reinterpret_cast<float4*>(stats)[t] = make_float4(M, L, R, tg);
+}
+
+// All ranges' statistics [n_shards, T, 4] -> lse, logp, entropy of the whole vocabulary.
+__global__ void shard_merge_kernel(const float* __restrict__ stats_all, int n_shards, const int32_t* __restrict__ ids,
+                                   int64_t T, int V_total, float* __restrict__ logp, float* __restrict__ lse,
+                                   float* __restrict__ entropy, uint32_t* __restrict__ status) {
+  const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (t >= T) return;
+  const float4* p4 = reinterpret_cast<const float4*>(stats_all);
+  float M = -CUDART_INF_F;
+  for (int s = 0; s < n_shards; ++s) M = fmaxf(M, p4[(int64_t)s * T + t].x);
+  float L = 0.f, R = 0.f, tg = 0.f;
+  for (int s = 0; s < n_shards; ++s) {
+    const float4 v = p4[(int64_t)s * T + t];
+    if (v.x > -CUDART_INF_F) {
+      const float w = expf(v.x - M);
+      L += v.y * w;
+      R += v.z * w;
+    }
+    tg += v.w;   // zero from every range but the one that owns the token
+  }
+  const float z = M + logf(L);
+  uint32_t bits = 0;
+  const int id = ids[t];
+  if (id < 0 || id >= V_total) { bits |= DRK_STATUS_BAD_ID; tg = 0.f; }
+  if (!isfinite(z)) bits |= DRK_STATUS_NONFINITE;
+  lse[t] = z;
+  logp[t] = tg - z;
+  if (entropy != nullptr) entropy[t] = z - R / L;
+  if (bits) atomicOr(status, bits);
+}
+
+int launch_shard_stats(const float* part, const float* tgt, const int32_t* ids, int id_off, int64_t T, int V,
+                       int nsplit, float* stats, uint32_t* status, cudaStream_t st) {
+  shard_stats_kernel<<<(unsigned)ceil_div(T, 256), 256, 0, st>>>(part, tgt, ids, id_off, T, V, nsplit, stats, status);
+  DRK_LAUNCHED();
+  return DRK_OK;
+}
+
+int launch_shard_merge(const float* stats_all, int n_shards, const int32_t* ids, int64_t T, int V_total, float* logp,
+                       float* lse, float* entropy, uint32_t* status, cudaStream_t st) {
+  shard_merge_kernel<<<(unsigned)ceil_div(T, 256), 256, 0, st>>>(stats_all, n_shards, ids, T, V_total, logp, lse,
+                                                                 entropy, status);
+  DRK_LAUNCHED();
+  return DRK_OK;
+}
+
 __global__ void f32_to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, size_t n) {
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += stride) dst[i] = __float2bfloat16(src[i]);
@@ -285,12 +354,14 @@ int launch_simt_fwd(const SimtFwdArgs& a, cudaStream_t st) {
   dim3 grid((unsigned)ceil_div(a.T, BM), (unsigned)a.nsplit);
   if (a.in_dtype == DRK_F32)
     lmhead_fwd_kernel<float><<<grid, kThreads, 0, st>>>((const float*)a.hidden, (const float*)a.W, a.ids, a.T,
-                                                        a.H, a.V, per, a.part, a.tgt);
+                                                        a.H, a.V, per, a.part, a.tgt, a.id_off);
   else
     lmhead_fwd_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)a.hidden,
                                                                 (const __nv_bfloat16*)a.W, a.ids, a.T, a.H,
-                                                                a.V, per, a.part, a.tgt);
+                                                                a.V, per, a.part, a.tgt, a.id_off);
   DRK_LAUNCHED();
+  if (a.stats != nullptr)
+    return launch_shard_stats(a.part, a.tgt, a.ids, a.id_off, a.T, a.V, a.nsplit, a.stats, a.status, st);
   return launch_lse_merge(a.part, a.tgt, a.ids, a.T, a.V, a.nsplit, a.logp, a.lse, a.entropy, a.status, nullptr,
                           nullptr, st);
 }
@@ -305,7 +376,7 @@ static int simt_bwd_typed(const SimtBwdArgs& a, cudaStream_t st) {
     const int vc_this = min(a.vc, a.V - v0);
     dim3 g1((unsigned)ceil_div(a.T, BM), (unsigned)ceil_div(vc_this, BN));
     lmhead_dl_kernel<TIn><<<g1, kThreads, 0, st>>>(hidden, W, a.ids, a.lse, a.coeff, a.T, a.H, a.V, v0, vc_this,
-                                                   a.vc, a.dL);
+                                                   a.vc, a.dL, a.id_off);
     DRK_LAUNCHED();
     // dW[v0:v0+vc_this, :] (+)= dL^T hidden      (M = v, N = h, K = t)
     dim3 g2((unsigned)ceil_div(vc_this, BM), (unsigned)ceil_div(a.H, BN));

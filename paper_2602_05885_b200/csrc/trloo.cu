@@ -96,4 +96,29 @@ int launch_trloo(const float* reward, const uint8_t* valid, const int32_t* promp
   return DRK_OK;
 }
 
+// Every turn of a trajectory is one training sample (Sec. 4.3): segment g of a packed micro-batch holds
+// turn seg_turn[g] of rollout seg_rollout[g] and takes that entry of the advantage table.
+__global__ void segment_advantages_kernel(const float* __restrict__ adv, const int32_t* __restrict__ seg_rollout,
+                                          const int32_t* __restrict__ seg_turn, int R, int Tmax, int S,
+                                          float* __restrict__ seg_adv, uint32_t* __restrict__ status) {
+  const int g = blockIdx.x * blockDim.x + threadIdx.x;
+  if (g >= S) return;
+  const int i = seg_rollout[g], t = seg_turn[g];
+  if (i < 0 || i >= R || t < 0 || t >= Tmax) {
+    seg_adv[g] = 0.f;
+    atomicOr(status, DRK_STATUS_BAD_SEGMENTS);
+    return;
+  }
+  seg_adv[g] = adv[(size_t)i * Tmax + t];
+}
+
+int launch_segment_advantages(const float* adv, const int32_t* seg_rollout, const int32_t* seg_turn, int R, int Tmax,
+                              int S, float* seg_adv, uint32_t* status, cudaStream_t st) {
+  if (S == 0) return DRK_OK;
+  segment_advantages_kernel<<<(unsigned)ceil_div(S, 256), 256, 0, st>>>(adv, seg_rollout, seg_turn, R, Tmax, S,
+                                                                        seg_adv, status);
+  DRK_LAUNCHED();
+  return DRK_OK;
+}
+
 }  // namespace drk

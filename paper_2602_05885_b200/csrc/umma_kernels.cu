@@ -58,6 +58,8 @@ struct UmmaParams {
   int64_t rows;  // valid extent of the tile-row index (T, or the chunk's width for DW)
   int cols;      // valid extent of the tile-column index (V, the chunk's width, or H)
   int v0;        // first vocabulary column of the chunk (0 for FWD)
+  int id_off;    // W holds columns [id_off, id_off + width) of a larger vocabulary: ids are taken relative to it
+  int id_width;  // number of columns W holds
   int64_t T;
   const int32_t* ids;
   const float* lse;
@@ -380,10 +382,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       int id = -1;
       float c_t = 0.f, z2 = 0.f;
       if constexpr (MODE == FWD) {
-        if (row_ok) id = p.ids[orow];   // partials and target logits stay indexed by the (compact) row
+        if (row_ok) id = local_id(p.ids[orow], p.id_off, p.id_width);   // partials and target logits stay indexed by the (compact) row
       }
       if constexpr (MODE == DL) {
-        if (row_ok && orow >= 0) { id = p.ids[orow]; c_t = p.coeff[orow]; z2 = p.lse[orow] * kLog2e; }
+        if (row_ok && orow >= 0) { id = local_id(p.ids[orow], p.id_off, p.id_width); c_t = p.coeff[orow]; z2 = p.lse[orow] * kLog2e; }
       }
       for (int n = un.n_begin; n < un.n_end; ++n) {
         const int acc = tc & 1;
@@ -679,11 +681,14 @@ int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st) {
   if (a.nsplit > 32 || a.nsplit * 8 >= p.n_tiles) p.group_m = panel_group(TM * ctas, a.H);  // short units: panel budget
   else p.group_m = slots / a.nsplit > 0 ? slots / a.nsplit : 1;                    // long ranges: one wave
   p.rows = a.T; p.cols = a.V; p.v0 = 0; p.T = a.T;
+  p.id_off = a.id_off; p.id_width = a.V;
   p.ids = a.ids; p.part = a.part; p.tgt = a.tgt; p.status = a.status;
-  p.want_entropy = a.entropy != nullptr;
+  p.want_entropy = a.entropy != nullptr || a.stats != nullptr;   // the statistics carry the same third sum
   p.rowmap = a.rowmap; p.n_rows = a.n_rows;
   int rc = launch_mode<FWD>(ctas, mh, mw, p, st);
   if (rc != DRK_OK) return rc;
+  if (a.stats != nullptr)
+    return launch_shard_stats(a.part, a.tgt, a.ids, a.id_off, a.T, a.V, a.nsplit, a.stats, a.status, st);
   return launch_lse_merge(a.part, a.tgt, a.ids, a.T, a.V, a.nsplit, a.logp, a.lse, a.entropy, a.status, a.rowmap,
                           a.n_rows, st);
 }
@@ -716,6 +721,7 @@ int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {
       p.k_blocks = (int)ceil_div(a.H, TK);
       p.nj = p.n_tiles; p.tiles_per_unit = 1; p.group_m = 16 / ctas;
       p.rows = a.T; p.cols = vc_this; p.v0 = v0; p.T = a.T;
+      p.id_off = a.id_off; p.id_width = a.V;
       p.ids = a.ids; p.lse = a.lse; p.coeff = a.coeff; p.dL = a.dL; p.vc = a.vc; p.status = a.status;
       p.rowmap = a.rowmap; p.n_rows = a.n_rows;
       int rc = launch_mode<DL>(ctas, mh_k, mw_k, p, st);

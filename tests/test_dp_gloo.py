@@ -1,8 +1,11 @@
-"""The data-parallel host logic on two gloo ranks (CPU): disjoint micro-batch ownership and the
-max-over-ranks time that defines whole-job throughput."""
+"""The multi-rank host logic on gloo ranks (CPU): disjoint micro-batch ownership and the max-over-ranks
+time that defines whole-job throughput; the two exchanges of the vocabulary-parallel form (all-gather of
+per-row statistics in rank order, all-reduce of the dH parts), with the oracle standing in for the
+kernels on each rank."""
 import os
 import socket
 
+import numpy as np
 import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
@@ -64,3 +67,62 @@ def test_assignment_balances_and_covers():
     tot = [sum(loads[i] for i in o) for o in owned]
     assert max(tot) - min(tot) <= 700
     assert dp.max_over_ranks(3.5) == 3.5 and dp.sum_over_ranks(2.0) == 2.0   # no process group: identity
+
+
+def _vocab_worker(rank, world, port, out):
+    from oracle import drk_oracle as O
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    rng = np.random.default_rng(5)                       # the same micro-batch on every rank
+    T, H, V = 12, 8, 700
+    hidden, W = rng.normal(size=(T, H)), rng.normal(size=(V, H))
+    ids = rng.integers(0, V, size=T)
+    coeff = rng.normal(size=T)
+    a, b = dp.vocab_shards(V, world)[rank]
+    s = O.logits(hidden, W)
+    stats = torch.from_numpy(O.shard_stats(s, ids, a, b))
+    stats_all = dp.all_gather_stats(stats)
+    assert stats_all.shape == (world, T, 4) and torch.equal(stats_all[rank], stats)
+    logp, lse, ent = O.merge_shard_stats(stats_all.numpy())
+    dH_part, dW_rows = O.shard_gradients(hidden, W, s, lse, ids, coeff, a, b)
+    dH = dp.all_reduce_dh(torch.from_numpy(dH_part.copy()))
+    out.put((rank, (a, b), logp, lse, dH.numpy(), dW_rows))
+    dist.destroy_process_group()
+
+
+def test_vocabulary_parallel_exchanges_on_three_ranks():
+    from oracle import drk_oracle as O
+    world = 3
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_vocab_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted((q.get(timeout=120) for _ in procs), key=lambda r: r[0])
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    rng = np.random.default_rng(5)
+    T, H, V = 12, 8, 700
+    hidden, W = rng.normal(size=(T, H)), rng.normal(size=(V, H))
+    ids = rng.integers(0, V, size=T)
+    coeff = rng.normal(size=T)
+    s = O.logits(hidden, W)
+    logp, lse = O.token_logprob(s, ids)
+    dH, dW = O.gradients(hidden, W, s, lse, ids, coeff)
+    ranges = [r[1] for r in res]
+    assert ranges == [(0, 256), (256, 512), (512, 700)]          # tiles of 256 rows, the last rank takes the rest
+    for _, _, lp, z, dh, _ in res:                                # identical, complete results on every rank
+        assert np.abs(lp - logp).max() < 1e-12 and np.abs(z - lse).max() < 1e-12
+        assert np.abs(dh - dH).max() < 1e-12
+    assert np.abs(np.concatenate([r[5] for r in res]) - dW).max() < 1e-12
+
+
+def test_vocab_shards_cover_the_vocabulary():
+    for V, world in ((151936, 8), (151936, 2), (151936, 1), (4096, 3), (300, 4)):
+        sh = dp.vocab_shards(V, world)
+        assert len(sh) == world and sh[0][0] == 0 and sh[-1][1] == V
+        assert all(a[1] == b[0] for a, b in zip(sh, sh[1:]))
+        assert all(a % 256 == 0 for a, _ in sh if a < V)
