@@ -401,7 +401,7 @@ def main():
     traffic = None
     if (args.workload, T, args.mrs, args.dw_dtype, args.dh_dtype, args.v_chunk, args.engine, args.forward_rows,
             args.parallelism) == ("qwen3-14b", 32768, "wide", "f32", "bf16", 0, "auto", "all", "data"):
-        traffic = 165.37e9
+        traffic = 181.81e9
     # the same call with rejection switched off: every loss-masked token goes through the backward
     p_off = B.drk_pg_params_default()
     ctypes_copy = [f[0] for f in p._fields_]
