@@ -312,6 +312,17 @@ int drk_pg_diagnostics(const float* logp, const float* rollout_logp, const float
                        const void* dH, int32_t dh_dtype, const void* dW, int32_t dw_dtype, int32_t H,
                        int32_t V, double* out, void* stream);
 
+/*
+ * Self-test of the library's failure handling (no counterpart in the paper).  Every on-chip wait of the
+ * tensor-core kernels is bounded: when one runs out, the block raises an abort flag that makes its other
+ * waiters leave, sets DRK_STATUS_TIMEOUT in the status word and returns, so the context stays usable.  This
+ * call launches one block that waits, through the same wait routines, on a barrier that nothing ever signals:
+ * one thread with the limit limit_ms (1..1000), one warp with the kernels' own limit (2 s) that must leave
+ * early on the abort flag.  Afterwards *status (device, OR-ed into) has DRK_STATUS_TIMEOUT set and waited_ns
+ * (device uint64[2]) holds how long the thread and the warp waited.  Nothing else is touched.
+ */
+int drk_selftest_bounded_wait(uint32_t limit_ms, uint32_t* status, uint64_t* waited_ns, void* stream);
+
 /* Number of kernels the last call on this host thread enqueued (0 after an error). */
 int drk_last_launch_count(void);
 

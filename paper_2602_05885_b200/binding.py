@@ -128,6 +128,8 @@ def load() -> ctypes.CDLL:
     lib.drk_pg_shard_loss_bwd.restype = ctypes.c_int
     lib.drk_segment_advantages.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp]
     lib.drk_segment_advantages.restype = ctypes.c_int
+    lib.drk_selftest_bounded_wait.argtypes = [ctypes.c_uint32, vp, vp, vp]
+    lib.drk_selftest_bounded_wait.restype = ctypes.c_int
     lib.drk_last_launch_count.argtypes = []
     lib.drk_last_launch_count.restype = ctypes.c_int
     lib.drk_status_string.argtypes = [ctypes.c_int]
@@ -298,6 +300,13 @@ def drk_segment_advantages(adv, seg_rollout, seg_turn, R: int, Tmax: int, S: int
                                        _ptr(status), _stream(stream))
     if check and rc != DRK_OK:
         raise DrkError(rc, "drk_segment_advantages")
+    return rc
+
+
+def drk_selftest_bounded_wait(limit_ms: int, status, waited_ns, stream=None, check: bool = True) -> int:
+    rc = load().drk_selftest_bounded_wait(limit_ms, _ptr(status), _ptr(waited_ns), _stream(stream))
+    if check and rc != DRK_OK:
+        raise DrkError(rc, "drk_selftest_bounded_wait")
     return rc
 
 

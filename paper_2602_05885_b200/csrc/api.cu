@@ -419,6 +419,16 @@ int drk_segment_advantages(const float* adv, const int32_t* seg_rollout, const i
   return rc;
 }
 
+int drk_selftest_bounded_wait(uint32_t limit_ms, uint32_t* status, uint64_t* waited_ns, void* stream) {
+  g_launches = 0;
+  if (limit_ms < 1 || limit_ms > 1000 || !status || !waited_ns) return DRK_ERR_INVALID_ARG;
+  int rc = check_arch();
+  if (rc != DRK_OK) return rc;
+  rc = launch_bounded_wait_selftest(limit_ms, status, waited_ns, static_cast<cudaStream_t>(stream));
+  if (rc != DRK_OK) g_launches = 0;
+  return rc;
+}
+
 int drk_last_launch_count(void) { return g_launches; }
 
 const char* drk_status_string(int s) {

@@ -121,6 +121,8 @@ int launch_compact(const CompactArgs& a, cudaStream_t st);
 // need[t] = 1 for loss-masked tokens inside a segment, else 0 (the rows whose log-prob the loss can use)
 int launch_need_rows(const uint8_t* loss_mask, const int32_t* cu, int64_t T, int S, float* need, cudaStream_t st);
 
+int launch_bounded_wait_selftest(uint32_t limit_ms, uint32_t* status, uint64_t* waited_ns, cudaStream_t st);
+
 // Small utility kernels.
 int launch_f32_to_bf16(const float* src, __nv_bfloat16* dst, size_t n, cudaStream_t st);
 

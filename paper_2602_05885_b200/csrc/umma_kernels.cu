@@ -506,6 +506,35 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   }
 }
 
+// Self-test of the bounded waits: one block waits on an mbarrier on which nothing ever arrives.  Lane 0 of
+// warp 0 waits like the producer and MMA threads do and gives up after limit_ns, raising the block's abort
+// flag; warp 1 waits like an epilogue warp (its own limit is WAIT_LIMIT_NS) and must leave as soon as it
+// sees the flag.  The block then reports DRK_STATUS_TIMEOUT exactly as the GEMM kernels do.
+__global__ void bounded_wait_selftest_kernel(uint32_t* status, uint64_t limit_ns, uint64_t* waited_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  const uint32_t bar_addr = ptx::smem_u32(&bar);
+  volatile int* abort = &abort_flag;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(bar_addr, 1);
+    *abort = 0;
+    ptx::fence_barrier_init();
+  }
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint64_t t0 = ptx::globaltimer_ns();
+  bool ok = true;
+  if (warp == 0) {
+    if (lane == 0) ok = ptx::mbar_wait(bar_addr, 0, abort, limit_ns);
+  } else {
+    ok = mbar_wait_warp(bar_addr, 0, abort, lane);
+  }
+  const uint64_t waited = ptx::globaltimer_ns() - t0;
+  if (lane == 0) waited_ns[warp] = waited;
+  __syncthreads();
+  if (threadIdx.x == 0 && (*abort || !ok)) atomicOr(status, DRK_STATUS_TIMEOUT);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
@@ -661,6 +690,12 @@ static int panel_group(int rows_per_tile, int64_t k_elems) {
   const double panel = (double)rows_per_tile * (double)k_elems * 2.0;
   int g = (int)(40.0 * 1024 * 1024 / panel);
   return g < 1 ? 1 : (g > 64 ? 64 : g);
+}
+
+int launch_bounded_wait_selftest(uint32_t limit_ms, uint32_t* status, uint64_t* waited_ns, cudaStream_t st) {
+  bounded_wait_selftest_kernel<<<1, 64, 0, st>>>(status, (uint64_t)limit_ms * 1000000ull, waited_ns);
+  DRK_LAUNCHED();
+  return DRK_OK;
 }
 
 int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st) {

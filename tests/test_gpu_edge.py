@@ -157,3 +157,25 @@ def test_large_logits_stay_finite_and_accurate(engine):
     ref = Hh.oracle_eval(case, *OPEN)
     assert Hh.rel_fro(Hh.f64(dev["dH"]), ref["dH"]) <= Hh.TOL_GRAD_FRO
     assert Hh.rel_fro(Hh.f64(dev["dW"]), ref["dW"]) <= Hh.TOL_GRAD_FRO
+
+
+def test_a_wait_that_runs_out_reports_a_timeout_and_leaves_the_context_usable():
+    # a barrier that nothing signals: the bounded wait gives up after its limit, the other waiter of the block
+    # leaves on the abort flag long before its own 2 s limit, and the status word says so
+    dev = torch.device("cuda:0")
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    waited = torch.zeros(2, dtype=torch.int64, device=dev)
+    B.drk_selftest_bounded_wait(50, status, waited)
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.DRK_STATUS_TIMEOUT
+    w = waited.tolist()
+    assert 50e6 <= w[0] < 150e6, w            # the limit, not more than a little beyond it
+    assert w[1] < 150e6, w                    # the warp did not sit out its own limit
+    assert B.drk_selftest_bounded_wait(0, status, waited, check=False) == B.DRK_ERR_INVALID_ARG
+    assert B.drk_selftest_bounded_wait(5000, status, waited, check=False) == B.DRK_ERR_INVALID_ARG
+    # the context is intact: an ordinary call right after it works
+    case = Hh.build_plain_case("after-timeout", T=300, H=64, V=700, dtype=torch.bfloat16, S=2, seed=3)
+    logp, lse, st = B.pg_logprob_fwd(case.hidden.to(dev), case.W.to(dev), case.ids.to(dev))
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    assert float((logp.double().cpu() - torch.from_numpy(case.logp)).abs().max()) <= Hh.TOL_LOGP_BF16
