@@ -178,3 +178,84 @@ def test_full_size_bench_inputs_sampled_rows(shape):
     scale = dW.double().abs().sum(dim=0)
     assert float((colsum.abs() / scale.clamp(min=1e-30)).max()) < 2e-3
     assert float(dW.abs().max()) > 0
+
+
+def test_full_size_vocabulary_parallel_two_ranges():
+    """The benchmark's 14B-shaped micro-batch with W split into the two row ranges `bench.py --parallelism vocab
+    --gpus 2` would use: sampled rows against the oracle (log-prob, lse, entropy from the recombined statistics;
+    dH from the summed parts), the zero-column-sum identity over both ranges' dW, and agreement of each range's
+    dW rows with the unsplit call."""
+    from paper_2602_05885_b200 import dp
+    dev = torch.device("cuda:0")
+    wl = workload.build("qwen3-14b", dev, seed=2000)
+    T, H, V, S = wl.T, wl.H, wl.V, wl.S
+    p = _bench_params(wl, mrs="off")
+    p.norm = B.DRK_NORM_EXPLICIT
+    p.explicit_scale = F32(1.0 / T)
+    p.dh_dtype = B.DRK_F32                                   # the parts are summed by the caller
+    g = torch.Generator().manual_seed(8)
+    seg_adv = torch.randn(S, generator=g).float().to(dev)
+    cuts = dp.vocab_shards(V, 2)
+    stats = []
+    for a, b in cuts:
+        n = B.drk_pg_workspace_bytes(T, H, b - a, 0, B.DRK_BF16, p, 0)
+        ws = torch.empty(n, dtype=torch.uint8, device=dev)
+        st = torch.empty((T, 4), device=dev)
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        B.drk_pg_shard_stats_fwd(wl.hidden, wl.W[a:b], B.DRK_BF16, wl.ids, T, H, b - a, a, V, p.engine, st, ws, n, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        stats.append(st)
+        del ws
+    stats_all = torch.stack(stats).contiguous()
+    dH = torch.zeros((T, H), dtype=torch.float32, device=dev)
+    dW_parts = []
+    first = None
+    for a, b in cuts:
+        bufs = B.PgLossBuffers(T, H, b - a, S, B.DRK_BF16, p, dev)
+        B.drk_pg_shard_loss_bwd(wl.hidden, wl.W[a:b], B.DRK_BF16, wl.ids, stats_all, len(cuts), wl.rollout_logp,
+                                wl.loss_mask, wl.cu, seg_adv, T, H, b - a, a, V, S, p, bufs.loss, bufs.logp, bufs.lse,
+                                bufs.entropy, bufs.seg_w, bufs.seg_keep, bufs.counters, bufs.dH, bufs.dW,
+                                bufs.workspace, bufs.workspace_bytes, bufs.status)
+        torch.cuda.synchronize()
+        assert int(bufs.status.item()) == 0
+        dH += bufs.dH
+        dW_parts.append(bufs.dW)
+        if first is None:
+            first = dict(logp=bufs.logp.clone(), lse=bufs.lse.clone(), entropy=bufs.entropy.clone(), loss=bufs.loss.clone())
+        else:
+            assert torch.equal(bufs.logp, first["logp"]) and torch.equal(bufs.loss, first["loss"])
+        bufs.workspace = None
+    mask = wl.loss_mask.cpu().numpy()
+    cu = wl.cu.cpu().numpy()
+    keep = np.array([mask[cu[j]:cu[j + 1]].any() for j in range(S)])
+    lr = O.coeff_and_loss(np.zeros(T), keep, mask, cu, Hh.f64(seg_adv), O.NORM_EXPLICIT, float(p.explicit_scale))
+    rng = np.random.default_rng(5)
+    sample = np.sort(rng.choice(T, size=192, replace=False))
+    st = torch.from_numpy(sample)
+    hid = Hh.f64(wl.hidden[st.to(dev)])
+    W64 = Hh.f64(wl.W.cpu())
+    ids = wl.ids.cpu().numpy().astype(np.int64)[sample]
+    s = O.logits(hid, W64)
+    logp, lse = O.token_logprob(s, ids)
+    assert np.abs(Hh.f64(first["logp"])[sample] - logp).max() <= Hh.TOL_LOGP_BF16
+    assert np.abs(Hh.f64(first["lse"])[sample] - lse).max() <= Hh.TOL_LOGP_BF16
+    assert np.abs(Hh.f64(first["entropy"])[sample] - O.token_entropy(s)).max() <= Hh.TOL_LOGP_BF16
+    for k, (a, b) in enumerate(cuts):                         # the ranges' statistics on the sampled rows
+        ref = O.shard_stats(s, ids, a, b)
+        got = Hh.f64(stats_all[k][st.to(dev)])
+        assert np.abs((got[:, 0] + np.log(got[:, 1])) - (ref[:, 0] + np.log(ref[:, 1]))).max() <= Hh.TOL_LOGP_BF16
+        assert np.abs(got[:, 3] - ref[:, 3]).max() <= Hh.TOL_LOGP_BF16
+    dH_s, _ = O.gradients(hid, W64, s, lse, ids, lr.coeff[sample])
+    assert Hh.rel_fro(Hh.f64(dH[st.to(dev)]), dH_s) <= Hh.TOL_GRAD_FRO
+    del W64, s
+    colsum = sum(d.double().sum(dim=0) for d in dW_parts)
+    scale = sum(d.double().abs().sum(dim=0) for d in dW_parts)
+    assert float((colsum.abs() / scale.clamp(min=1e-30)).max()) < 2e-3
+    # against the unsplit call on the same inputs
+    p.dh_dtype = B.DRK_BF16
+    whole = _run(wl, p, seg_adv)
+    for (a, b), d in zip(cuts, dW_parts):
+        diff = (d - whole.dW[a:b]).double().norm() / whole.dW[a:b].double().norm()
+        assert float(diff) <= 1e-3
+    assert float((dH - whole.dH.float()).double().norm() / whole.dH.double().norm()) <= 1e-2
