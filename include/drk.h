@@ -289,6 +289,11 @@ int drk_pg_shard_stats_fwd(const void* hidden, const void* W_shard, int32_t in_d
                            int64_t T, int32_t H, int32_t V_local, int32_t v_begin, int32_t V_total,
                            int32_t engine, float* stats, void* workspace, size_t workspace_bytes,
                            uint32_t* status, void* stream);
+/* Step 3 without loss and gradients: log-probs, lse and (entropy may be NULL) entropy from all ranges'
+ * statistics, i.e. drk_pg_logprob_fwd for a vocabulary-split LM head.  All pointers device. */
+int drk_pg_shard_merge(const float* stats_all, int32_t n_shards, const int32_t* ids, int64_t T,
+                       int32_t V_total, float* logp, float* lse, float* entropy, uint32_t* status,
+                       void* stream);
 int drk_pg_shard_loss_bwd(const void* hidden, const void* W_shard, int32_t in_dtype, const int32_t* ids,
                           const float* stats_all, int32_t n_shards, const float* rollout_logp,
                           const uint8_t* loss_mask, const int32_t* cu_seqlens, const float* seg_adv,

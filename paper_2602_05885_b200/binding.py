@@ -126,6 +126,8 @@ def load() -> ctypes.CDLL:
                                           ctypes.POINTER(drk_pg_params), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz,
                                           vp, vp]
     lib.drk_pg_shard_loss_bwd.restype = ctypes.c_int
+    lib.drk_pg_shard_merge.argtypes = [vp, i32, vp, i64, i32, vp, vp, vp, vp, vp]
+    lib.drk_pg_shard_merge.restype = ctypes.c_int
     lib.drk_segment_advantages.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp]
     lib.drk_segment_advantages.restype = ctypes.c_int
     lib.drk_selftest_bounded_wait.argtypes = [ctypes.c_uint32, vp, vp, vp]
@@ -276,6 +278,15 @@ def drk_pg_shard_stats_fwd(hidden, W_shard, in_dtype: int, ids, T: int, H: int, 
                                        _stream(stream))
     if check and rc != DRK_OK:
         raise DrkError(rc, "drk_pg_shard_stats_fwd")
+    return rc
+
+
+def drk_pg_shard_merge(stats_all, n_shards: int, ids, T: int, V_total: int, logp, lse, entropy, status, stream=None,
+                       check: bool = True) -> int:
+    rc = load().drk_pg_shard_merge(_ptr(stats_all), n_shards, _ptr(ids), T, V_total, _ptr(logp), _ptr(lse),
+                                   _ptr(entropy), _ptr(status), _stream(stream))
+    if check and rc != DRK_OK:
+        raise DrkError(rc, "drk_pg_shard_merge")
     return rc
 
 

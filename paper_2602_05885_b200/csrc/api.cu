@@ -2,6 +2,7 @@
 #include "common.cuh"
 #include <cmath>
 #include <limits>
+#include <nvtx3/nvToolsExt.h>   // header-only; ranges cost nothing unless a profiler is attached
 
 namespace drk {
 
@@ -10,6 +11,14 @@ thread_local int g_launches = 0;
 namespace {
 
 constexpr int kDefaultVChunk = 8192;
+
+// Names a phase of the fused call on the profiler's timeline for as long as the object lives.
+struct Range {
+  explicit Range(const char* name) { nvtxRangePushA(name); }
+  ~Range() { nvtxRangePop(); }
+  Range(const Range&) = delete;
+  Range& operator=(const Range&) = delete;
+};
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
@@ -204,11 +213,14 @@ int loss_fwd_bwd_impl(const void* hidden, const void* W, int32_t in_dtype, const
 
   auto fail = [&](int code) { g_launches = 0; return code; };
 
+  Range call_range(sh ? "drk_pg_shard_loss_bwd" : "drk_pg_loss_fwd_bwd");
   if (T > 0 && sh != nullptr) {
+    Range r("drk: recombine range statistics");
     rc = launch_shard_merge(sh->stats_all, sh->n_shards, ids, T, sh->V_total, logp, lse, entropy, status, st);
     if (rc != DRK_OK) return fail(rc);
   } else if (T > 0 && p.forward_rows == 1 && !simt) {
     // forward over the rows the loss can use: loss-masked tokens inside segments; the rest read 0
+    Range r("drk: forward (usable rows)");
     rc = launch_need_rows(loss_mask, cu_seqlens, T, S, bw.coeff, st);
     if (rc != DRK_OK) return fail(rc);
     CompactArgs ca{bw.coeff, static_cast<const __nv_bfloat16*>(hidden), T, H, bw.blk_cnt, bw.blk_off, bw.n_rows,
@@ -223,20 +235,25 @@ int loss_fwd_bwd_impl(const void* hidden, const void* W, int32_t in_dtype, const
                  bw.rowmap, bw.n_rows);
     if (rc != DRK_OK) return fail(rc);
   } else if (T > 0) {
+    Range r("drk: forward");
     rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, p.engine, fw, logp, lse, entropy, status, st);
     if (rc != DRK_OK) return fail(rc);
   }
-  MrsArgs m{};
-  m.logp = logp; m.rollout_logp = rollout_logp; m.loss_mask = loss_mask; m.cu = cu_seqlens; m.seg_adv = seg_adv;
-  m.T = T; m.S = S;
-  m.ln_lo = p.mrs_lo > 0.f ? std::log((double)p.mrs_lo) : -std::numeric_limits<double>::infinity();
-  m.ln_hi = std::isinf(p.mrs_hi) ? std::numeric_limits<double>::infinity() : std::log((double)p.mrs_hi);
-  m.ln_veto = p.veto_ratio > 0.f ? std::log((double)p.veto_ratio) : -std::numeric_limits<double>::infinity();
-  m.norm = p.norm; m.explicit_scale = p.explicit_scale; m.keep_from_caller = p.keep_from_caller;
-  m.seg_w = seg_w; m.seg_keep = seg_keep; m.loss = loss; m.counters = counters; m.coeff = bw.coeff;
-  m.seg_stats = bw.seg_stats; m.status = status;
-  rc = launch_mrs(m, st);
+  {
+    Range r("drk: rejection sampling, coefficients, loss");
+    MrsArgs m{};
+    m.logp = logp; m.rollout_logp = rollout_logp; m.loss_mask = loss_mask; m.cu = cu_seqlens; m.seg_adv = seg_adv;
+    m.T = T; m.S = S;
+    m.ln_lo = p.mrs_lo > 0.f ? std::log((double)p.mrs_lo) : -std::numeric_limits<double>::infinity();
+    m.ln_hi = std::isinf(p.mrs_hi) ? std::numeric_limits<double>::infinity() : std::log((double)p.mrs_hi);
+    m.ln_veto = p.veto_ratio > 0.f ? std::log((double)p.veto_ratio) : -std::numeric_limits<double>::infinity();
+    m.norm = p.norm; m.explicit_scale = p.explicit_scale; m.keep_from_caller = p.keep_from_caller;
+    m.seg_w = seg_w; m.seg_keep = seg_keep; m.loss = loss; m.counters = counters; m.coeff = bw.coeff;
+    m.seg_stats = bw.seg_stats; m.status = status;
+    rc = launch_mrs(m, st);
+  }
   if (rc != DRK_OK) return fail(rc);
+  Range bwd_range("drk: backward");
 
   if (T == 0) {
     // no tokens: gradients are zero
@@ -388,6 +405,21 @@ int drk_pg_shard_stats_fwd(const void* hidden, const void* W_shard, int32_t in_d
   const FwdWs w = carve_fwd(c, T, V_local, simt, engine);
   rc = run_fwd(hidden, W_shard, in_dtype, ids, T, H, V_local, simt, engine, w, nullptr, nullptr, nullptr, status,
                static_cast<cudaStream_t>(stream), nullptr, nullptr, nullptr, v_begin, stats);
+  if (rc != DRK_OK) g_launches = 0;
+  return rc;
+}
+
+int drk_pg_shard_merge(const float* stats_all, int32_t n_shards, const int32_t* ids, int64_t T, int32_t V_total,
+                       float* logp, float* lse, float* entropy, uint32_t* status, void* stream) {
+  g_launches = 0;
+  if (T < 0 || T > (1 << 24) || V_total < 1 || V_total > (1 << 24) || n_shards < 1 || n_shards > 4096)
+    return DRK_ERR_INVALID_ARG;
+  if (T == 0) return DRK_OK;
+  if (!stats_all || !ids || !logp || !lse || !status || !aligned(stats_all, 16)) return DRK_ERR_INVALID_ARG;
+  int rc = check_arch();
+  if (rc != DRK_OK) return rc;
+  rc = launch_shard_merge(stats_all, n_shards, ids, T, V_total, logp, lse, entropy, status,
+                          static_cast<cudaStream_t>(stream));
   if (rc != DRK_OK) g_launches = 0;
   return rc;
 }

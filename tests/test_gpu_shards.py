@@ -50,6 +50,13 @@ def run_sharded(case, cuts, p, dev=torch.device("cuda:0")):
         assert int(bufs.status.item()) == 0
         outs.append(bufs)
     first = outs[0]
+    # the forward-only recombination gives the same log-probs, lse and entropy as the loss call
+    lp, z, ent = (torch.full((T,), float("nan"), device=dev) for _ in range(3))
+    st_word = torch.zeros(1, dtype=torch.int32, device=dev)
+    B.drk_pg_shard_merge(stats_all, len(cuts), ids, T, V, lp, z, ent, st_word)
+    torch.cuda.synchronize()
+    assert int(st_word.item()) == 0
+    assert torch.equal(lp, first.logp) and torch.equal(z, first.lse) and torch.equal(ent, first.entropy)
     for o in outs[1:]:        # what is not a gradient is identical on every rank, bit for bit
         for name in ("loss", "logp", "lse", "entropy", "seg_w", "seg_keep", "counters"):
             assert torch.equal(getattr(o, name), getattr(first, name)), name
