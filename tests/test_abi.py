@@ -83,6 +83,41 @@ def test_validation_precedes_any_cuda_call():
     assert B.drk_last_launch_count() == 0
 
 
+def test_validation_of_the_vocabulary_range_calls_and_the_gather():
+    big = torch.zeros(256)
+    off = (-big.data_ptr() % 256) // 4
+    z = big[off:off + 64]                                    # 256-byte aligned, as a workspace must be
+    p = B.drk_pg_params_default()
+    fwd = lambda V_local, v_begin, V_total, T=8, H=8: B.drk_pg_shard_stats_fwd(
+        z, z, B.DRK_BF16, z, T, H, V_local, v_begin, V_total, 0, z, z, 1 << 20, z, stream=0, check=False)
+    assert fwd(16, 8, 16) == B.DRK_ERR_INVALID_ARG          # the range leaves the vocabulary
+    assert fwd(16, -1, 64) == B.DRK_ERR_INVALID_ARG
+    assert fwd(0, 0, 64) == B.DRK_ERR_INVALID_ARG
+    assert fwd(16, 0, (1 << 24) + 1) == B.DRK_ERR_INVALID_ARG
+    assert fwd(16, 0, 64, T=0) == B.DRK_OK                  # nothing to do, nothing enqueued
+    bwd = lambda n_shards, v_begin, V_total, pp=p: B.drk_pg_shard_loss_bwd(
+        z, z, B.DRK_BF16, z, z, n_shards, z, z, z, z, 8, 8, 16, v_begin, V_total, 1, pp, z, z, z, z, z, z, z, z, z, z,
+        1 << 20, z, stream=0, check=False)
+    assert bwd(0, 0, 64) == B.DRK_ERR_INVALID_ARG
+    assert bwd(4097, 0, 64) == B.DRK_ERR_INVALID_ARG
+    assert bwd(2, 56, 64) == B.DRK_ERR_INVALID_ARG
+    p2 = B.drk_pg_params_default()
+    p2.forward_rows = 1
+    assert bwd(2, 0, 64, p2) == B.DRK_ERR_UNSUPPORTED        # no forward pass to restrict
+    merge = lambda n, T, V: B.drk_pg_shard_merge(z, n, z, T, V, z, z, None, z, stream=0, check=False)
+    assert merge(0, 8, 64) == B.DRK_ERR_INVALID_ARG and merge(2, -1, 64) == B.DRK_ERR_INVALID_ARG
+    assert merge(2, 8, 0) == B.DRK_ERR_INVALID_ARG and merge(2, 0, 64) == B.DRK_OK
+    assert B.drk_pg_shard_merge(None, 2, z, 8, 64, z, z, None, z, stream=0, check=False) == B.DRK_ERR_INVALID_ARG
+    gather = lambda R, Tmax, S, a=z: B.drk_segment_advantages(a, z, z, R, Tmax, S, z, z, stream=0, check=False)
+    assert gather(-1, 2, 4) == B.DRK_ERR_INVALID_ARG and gather(2, 2, -4) == B.DRK_ERR_INVALID_ARG
+    assert gather(2, 2, 0) == B.DRK_OK
+    assert gather(2, 2, 4, None) == B.DRK_ERR_INVALID_ARG
+    st = torch.zeros(4)
+    assert B.drk_selftest_bounded_wait(0, st, st, stream=0, check=False) == B.DRK_ERR_INVALID_ARG
+    assert B.drk_selftest_bounded_wait(1001, st, st, stream=0, check=False) == B.DRK_ERR_INVALID_ARG
+    assert B.drk_last_launch_count() == 0
+
+
 @pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-GPU behaviour")
 def test_without_a_gpu_calls_fail_loudly():
     # well-formed arguments, but no device: an error code, never a CPU fallback
