@@ -179,3 +179,18 @@ def test_a_wait_that_runs_out_reports_a_timeout_and_leaves_the_context_usable():
     torch.cuda.synchronize()
     assert int(st.item()) == 0
     assert float((logp.double().cpu() - torch.from_numpy(case.logp)).abs().max()) <= Hh.TOL_LOGP_BF16
+
+
+@pytest.mark.parametrize("T,H,V,S", [(200000, 64, 520, 40), (96, 64, 600000, 3)],
+                         ids=["many-rows", "wide-vocabulary"])
+def test_extreme_aspect_ratios(T, H, V, S):
+    # far more row tiles than the benchmark shapes have (index arithmetic past 2^17 rows, hundreds of compaction
+    # blocks), and a vocabulary four times the benchmark's with a handful of rows (thousands of vocabulary tiles,
+    # dozens of chunks)
+    case = Hh.build_plain_case("aspect", T=T, H=H, V=V, dtype=torch.bfloat16, S=S, seed=T % 97, mask_frac=0.25)
+    lo, hi = Hh.wide_band(case)
+    veto = float(np.float32(1e-4))
+    for engine in (B.DRK_ENGINE_AUTO, B.DRK_ENGINE_UMMA_1CTA):
+        dev = run_device(case, make_params(lo, hi, veto, engine=engine, dh_dtype=B.DRK_BF16))
+        assert dev["status"] == 0
+        Hh.check_against_oracle(case, dev, lo, hi, veto)
