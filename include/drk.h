@@ -157,6 +157,11 @@ typedef struct {
                             while later chunks are still being computed (the gradient exchange itself is the
                             trainer's; this library makes no collective call)                            */
   int32_t n_dw_chunk_events; /* must equal the chunk count when dw_chunk_events is given                    */
+  int32_t reuse_forward; /* 0: the call computes logp, lse (and entropy).  1: logp and lse are INPUTS, as written by
+                            an earlier drk_pg_logprob_fwd (or fused call) on the same hidden, W and ids, and the
+                            forward pass is skipped: a caller that judged its samples on log-probs from a
+                            separate forward (samples split over micro-batches) pays for the logits three times,
+                            not four.  entropy is left untouched.  forward_rows must be 0                 */
 } drk_pg_params;
 
 void drk_pg_params_default(drk_pg_params* p); /* host pointer */

@@ -55,6 +55,7 @@ class drk_pg_params(ctypes.Structure):
         ("forward_rows", ctypes.c_int32),
         ("dw_chunk_events", ctypes.POINTER(ctypes.c_void_p)),
         ("n_dw_chunk_events", ctypes.c_int32),
+        ("reuse_forward", ctypes.c_int32),
     ]
 
 

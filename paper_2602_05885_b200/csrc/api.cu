@@ -140,6 +140,8 @@ bool params_ok(const drk_pg_params& p) {
   if (p.v_chunk < 0) return false;
   if (p.keep_from_caller < 0 || p.keep_from_caller > 2) return false;
   if (p.forward_rows != 0 && p.forward_rows != 1) return false;
+  if (p.reuse_forward != 0 && p.reuse_forward != 1) return false;
+  if (p.reuse_forward == 1 && p.forward_rows != 0) return false;
   if (p.n_dw_chunk_events < 0 || (p.dw_chunk_events == nullptr && p.n_dw_chunk_events != 0)) return false;
   if (std::isnan(p.mrs_lo) || std::isnan(p.mrs_hi) || std::isnan(p.veto_ratio)) return false;
   if (p.norm == DRK_NORM_EXPLICIT && !std::isfinite(p.explicit_scale)) return false;
@@ -214,7 +216,9 @@ int loss_fwd_bwd_impl(const void* hidden, const void* W, int32_t in_dtype, const
   auto fail = [&](int code) { g_launches = 0; return code; };
 
   Range call_range(sh ? "drk_pg_shard_loss_bwd" : "drk_pg_loss_fwd_bwd");
-  if (T > 0 && sh != nullptr) {
+  if (T > 0 && sh == nullptr && p.reuse_forward == 1) {
+    // logp and lse come from an earlier forward over the same operands
+  } else if (T > 0 && sh != nullptr) {
     Range r("drk: recombine range statistics");
     rc = launch_shard_merge(sh->stats_all, sh->n_shards, ids, T, sh->V_total, logp, lse, entropy, status, st);
     if (rc != DRK_OK) return fail(rc);
@@ -306,6 +310,7 @@ void drk_pg_params_default(drk_pg_params* p) {
   p->forward_rows = 0;
   p->dw_chunk_events = nullptr;
   p->n_dw_chunk_events = 0;
+  p->reuse_forward = 0;
 }
 
 int drk_pg_bwd_chunks(int64_t T, int32_t H, int32_t V, int32_t in_dtype, const drk_pg_params* pp, int32_t* v_chunk) {

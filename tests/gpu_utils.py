@@ -7,7 +7,8 @@ from paper_2602_05885_b200 import binding as B
 
 
 def make_params(lo=None, hi=None, veto=None, norm=0, explicit_scale=1.0, dw_dtype=B.DRK_F32, dh_dtype=B.DRK_F32,
-                dw_accumulate=0, engine=B.DRK_ENGINE_AUTO, v_chunk=0, keep_from_caller=0, forward_rows=0):
+                dw_accumulate=0, engine=B.DRK_ENGINE_AUTO, v_chunk=0, keep_from_caller=0, forward_rows=0,
+                reuse_forward=0):
     p = B.drk_pg_params_default()
     if lo is not None:
         p.mrs_lo = lo
@@ -24,10 +25,11 @@ def make_params(lo=None, hi=None, veto=None, norm=0, explicit_scale=1.0, dw_dtyp
     p.v_chunk = v_chunk
     p.keep_from_caller = keep_from_caller
     p.forward_rows = forward_rows
+    p.reuse_forward = reuse_forward
     return p
 
 
-def run_device(case, p, seg_adv=None, dW_init=None, device="cuda:0", keep_in=None):
+def run_device(case, p, seg_adv=None, dW_init=None, device="cuda:0", keep_in=None, logp_in=None, lse_in=None):
     dev = torch.device(device)
     hidden = case.hidden.to(dev)
     W = case.W.to(dev)
@@ -44,6 +46,9 @@ def run_device(case, p, seg_adv=None, dW_init=None, device="cuda:0", keep_in=Non
     if dW_init is None:
         bufs.dW.fill_(float("nan"))
     bufs.logp.fill_(float("nan"))
+    if logp_in is not None:
+        bufs.logp.copy_(logp_in.to(dev))
+        bufs.lse.copy_(lse_in.to(dev))
     if keep_in is not None:
         bufs.seg_keep.copy_(keep_in.to(dev))
     B.pg_loss_fwd_bwd(hidden, W, ids, rl, mask, cu, adv, p, bufs)

@@ -230,3 +230,26 @@ def test_caller_retention_combined_with_mrs():
     assert dev["counters"][0] == ref["kept_tokens"] and dev["counters"][2] == ref["kept_segs"]
     assert Hh.rel_fro(Hh.f64(dev["dH"]), ref["dH"]) <= Hh.TOL_GRAD_FRO
     assert Hh.rel_fro(Hh.f64(dev["dW"]), ref["dW"]) <= Hh.TOL_GRAD_FRO
+
+
+@pytest.mark.parametrize("engine", [B.DRK_ENGINE_AUTO, B.DRK_ENGINE_SIMT])
+def test_reusing_an_earlier_forward(engine):
+    # samples judged on log-probs from a separate forward call: the fused call takes logp and lse as inputs and
+    # skips its own forward; everything it returns equals the ordinary call's, bit for bit
+    case = get_case("medium")
+    lo, hi = Hh.wide_band(case)
+    p = make_params(lo, hi, PAPER[2], engine=engine, v_chunk=2048)
+    whole = run_device(case, p)
+    d = torch.device("cuda:0")
+    logp, lse, st = B.pg_logprob_fwd(case.hidden.to(d), case.W.to(d), case.ids.to(d), engine=engine)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0 and torch.equal(logp.cpu(), whole["logp"])
+    again = run_device(case, make_params(lo, hi, PAPER[2], engine=engine, v_chunk=2048, reuse_forward=1),
+                       logp_in=logp, lse_in=lse)
+    for name in ("logp", "lse", "seg_w", "seg_keep", "counters", "loss", "dH", "dW"):
+        assert torch.equal(again[name], whole[name]), name
+    assert again["launches"] == whole["launches"] - 2           # no forward kernel, no merge
+    Hh.check_against_oracle(case, {k: v for k, v in again.items() if k != "entropy"}, lo, hi, PAPER[2])
+    # a restricted forward makes no sense together with no forward
+    bad = make_params(lo, hi, PAPER[2], reuse_forward=1, forward_rows=1)
+    assert B.drk_pg_workspace_bytes(case.T, case.H, case.V, case.S, B.DRK_BF16, bad, 1) == 0
