@@ -253,3 +253,41 @@ def test_reusing_an_earlier_forward(engine):
     # a restricted forward makes no sense together with no forward
     bad = make_params(lo, hi, PAPER[2], reuse_forward=1, forward_rows=1)
     assert B.drk_pg_workspace_bytes(case.T, case.H, case.V, case.S, B.DRK_BF16, bad, 1) == 0
+
+
+def test_gradient_accumulation_over_the_micro_batches_of_one_rollout_batch():
+    # TRLOO once over the whole rollout batch (on the device), then every packed micro-batch through the fused
+    # call with dW accumulating and one explicit normaliser for all of them, as a trainer would do; the
+    # accumulated dW must match the sum of the oracle's per-micro-batch gradients, the losses add up likewise
+    d = torch.device("cuda:0")
+    kw = dict(H=512, V=4200, dtype=torch.bfloat16, P=6, K=4, Tmax=3, len_lo=32, len_hi=200, capacity=900, seed=77,
+              sigma=0.05)
+    from paper_2602_05885_b200 import synth
+    rb = synth.rollout_batch(kw["P"], kw["K"], kw["Tmax"], kw["len_lo"], kw["len_hi"], kw["seed"])
+    n_mb = len(synth.pack_first_fit(rb, kw["capacity"]))
+    assert n_mb >= 3
+    cases = [Hh.build_case(f"mb{i}", microbatch=i, **kw) for i in range(n_mb)]
+    _, adv, _ = B.trloo_advantage(rb.reward.to(d), rb.valid.to(d), rb.prompt_of_rollout.to(d))
+    scale = F32(1.0 / sum(int(c.loss_mask.sum()) for c in cases))
+    open_band = (0.0, math.inf, 0.0)
+    dW_acc = torch.zeros((kw["V"], kw["H"]), dtype=torch.float32)
+    dW_ref = np.zeros((kw["V"], kw["H"]))
+    loss_dev = loss_ref = 0.0
+    for c in cases:
+        # every micro-batch uses the same W (the generator draws it from the seed alone)
+        assert torch.equal(c.W, cases[0].W)
+        seg_adv = torch.empty(c.S, dtype=torch.float32, device=d)
+        st = torch.zeros(1, dtype=torch.int32, device=d)
+        B.drk_segment_advantages(adv, c.seg_rollout.to(torch.int32).to(d), c.seg_turn.to(torch.int32).to(d),
+                                 adv.shape[0], adv.shape[1], c.S, seg_adv, st)
+        p = make_params(*open_band, norm=B.DRK_NORM_EXPLICIT, explicit_scale=scale, dw_accumulate=1, v_chunk=2048)
+        dev = run_device(c, p, seg_adv=seg_adv.cpu(), dW_init=dW_acc)
+        assert dev["status"] == 0 and int(st.item()) == 0
+        ref = Hh.check_against_oracle(c, dev, *open_band, norm=2, explicit_scale=scale, seg_adv=seg_adv.cpu(),
+                                      dW_before=Hh.f64(dW_acc))
+        dW_acc = dev["dW"]
+        dW_ref += ref["dW"]
+        loss_dev += float(dev["loss"])
+        loss_ref += ref["loss"]
+    assert Hh.rel_fro(Hh.f64(dW_acc), dW_ref) <= Hh.TOL_GRAD_FRO
+    assert abs(loss_dev - loss_ref) <= Hh.TOL_LOSS_REL * max(abs(loss_ref), 1e-3)
