@@ -146,6 +146,8 @@ def load() -> ctypes.CDLL:
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
     if t is None:
         return None
+    if not t.is_contiguous():
+        raise ValueError("the C ABI takes dense row-major arrays: pass a contiguous tensor")
     return t.data_ptr() if t.numel() > 0 else (t.data_ptr() or None)
 
 

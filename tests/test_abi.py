@@ -127,3 +127,12 @@ def test_without_a_gpu_calls_fail_loudly():
     assert rc in (B.DRK_ERR_CUDA, B.DRK_ERR_ARCH)
     with pytest.raises(B.DrkError):
         B.drk_trloo_advantage(z, z, z, 2, 2, 1.0, 0, z, z, z, stream=0)
+
+
+def test_binding_rejects_strided_tensors():
+    # the C ABI knows nothing of strides: a transposed or sliced-by-column tensor must not be passed silently
+    z = torch.zeros((8, 8))
+    with pytest.raises(ValueError):
+        B.drk_trloo_advantage(z.t(), z, z, 2, 2, 1.0, 0, z, z, z, stream=0, check=False)
+    with pytest.raises(ValueError):
+        B.drk_segment_advantages(z[:, ::2], z, z, 2, 2, 1, z, z, stream=0, check=False)
