@@ -517,6 +517,7 @@ def main():
                                           "tokens_per_s": T / (off_ms * 1e-3)},
                          "peak_source": f"bf16_tflops_sustained of {peaks['source']}",
                          "frac_of_burst": achieved / peaks["burst"], "frac_of_nominal_2250": achieved / 2250.0},
+            "value_no_rejection": T / (off_ms * 1e-3),   # the fused call alone with every sample retained (all rows in the backward)
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": n_launch, "clocks": clocks,
             "status_word": status, "counters": {"kept_tokens": counters[0], "masked_tokens": counters[1],
                                                 "kept_segments": counters[2], "vetoed_segments": counters[3]},
