@@ -94,7 +94,7 @@ def run_reference(args):
         return
     import numpy as np
     from oracle import drk_oracle as O
-    from paper_2602_05885_b200 import workload
+    from benchlib import workload
     try:
         from threadpoolctl import threadpool_info
         cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
@@ -138,7 +138,7 @@ def cpu_baseline(n_tok: int):
     """The oracle timed once on a bounded sample of the same workload (host cores of this machine)."""
     import numpy as np
     from oracle import drk_oracle as O
-    from paper_2602_05885_b200 import workload
+    from benchlib import workload
     try:
         from threadpoolctl import threadpool_info
         cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
@@ -162,7 +162,7 @@ def cpu_baseline(n_tok: int):
 def run_sweep(args):
     """Roofline sweep: T x V x H grid, bf16, equal-length segments, uniform ids.  One JSON line per point."""
     from paper_2602_05885_b200 import binding as B
-    from paper_2602_05885_b200 import workload
+    from benchlib import workload
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
     peaks = measured_peaks()
@@ -248,7 +248,8 @@ def main():
         return
 
     from paper_2602_05885_b200 import binding as B
-    from paper_2602_05885_b200 import dp, workload
+    from paper_2602_05885_b200 import dp
+    from benchlib import workload
     import torch.distributed as dist
 
     world = int(os.environ.get("WORLD_SIZE", "1"))

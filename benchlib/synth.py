@@ -254,3 +254,20 @@ def pick_outlier_segments(S: int, frac: float, seed: int) -> torch.Tensor:
     g = _gen(seed, "cpu")
     n = max(1, int(round(S * frac))) if S > 0 else 0
     return torch.randperm(S, generator=g)[:n]
+
+
+def threshold_between(values, spread: int = 2) -> float:
+    """A threshold that splits `values` about in half without sitting on any of them: the midpoint of the
+    widest gap between adjacent order statistics among the `spread` gaps either side of the median (fewer
+    for short lists: one gap per eight values)."""
+    a = sorted(float(v) for v in values)
+    n = len(a)
+    if n == 0:
+        return 1e-3
+    if n == 1:
+        return 2.0 * a[0] if a[0] > 0 else 1e-3
+    mid = n // 2
+    spread = min(spread, n // 8)
+    ks = range(max(0, mid - 1 - spread), min(n - 2, mid - 1 + spread) + 1)
+    k = max(ks, key=lambda i: (a[i + 1] - a[i], -abs(i - (mid - 1))))
+    return 0.5 * (a[k] + a[k + 1])

@@ -47,7 +47,8 @@ class Workload:
     n_microbatches: int = 1
 
     def wide_band(self):
-        """(lo, hi) = exp(-+q), q = median over segments of |mean noise|: about half the samples pass."""
+        """(lo, hi) = exp(-+q) with q between two adjacent order statistics of the segments' |mean noise| next
+        to their median: about half the samples pass, and no sample's mean lies on a threshold."""
         cu = self.cu.tolist()
         m = self.loss_mask.bool()
         vals = []
@@ -55,7 +56,7 @@ class Workload:
             sel = m[cu[j]:cu[j + 1]]
             if int(sel.sum()) > 0:
                 vals.append(abs(float(self.noise[cu[j]:cu[j + 1]][sel].mean())))
-        q = sorted(vals)[len(vals) // 2] if vals else 1e-3
+        q = synth.threshold_between(vals)
         return math.exp(-q), math.exp(q)
 
 

@@ -212,15 +212,18 @@ int drk_pg_logprob_fwd(const void* hidden, const void* W, int32_t in_dtype, cons
  * packaging variant of the forward call above.)  The scratch (per-row partial max / sum-exp pairs and
  * target logits) lives in a fixed array inside the library image instead:
  *   - every GPU on which the library is loaded holds DRK_NOALLOC_SCRATCH_BYTES until the process exits;
- *   - if the sizes need more (roughly 16*nsplit*T + 4*T bytes, nsplit <= 32 chosen from T and V) the call
- *     returns DRK_ERR_WORKSPACE and enqueues nothing; T = 32768 at H = 5120, V = 151936 needs about 2.2 MB;
+ *   - if the sizes need more (roughly 16*nsplit*T + 4*T bytes; nsplit, the number of vocabulary ranges per
+ *     row tile, is chosen from T and V and is at most 32 for the tensor-core engines and at most 64 for fp32
+ *     inputs or DRK_ENGINE_SIMT) the call returns DRK_ERR_WORKSPACE and enqueues nothing; T = 32768 at
+ *     H = 5120, V = 151936 needs about 2.2 MB;
  *   - the array is shared by all calls on a device and keeps the last call's contents.  What the
  *     computation reads is rewritten or cleared by each call, so consecutive calls on one stream are
  *     independent; calls that may run concurrently on the GPU (unordered streams) race on it;
  *   - the first call on each device looks up the array's device address.  Make that first call
  *     outside any stream capture.
  * It calls no cudaMalloc / cudaFree and no allocating library routine.  Arguments, outputs, status bits
- * and return codes are those of drk_pg_logprob_fwd, without the workspace pair.
+ * and return codes are those of drk_pg_logprob_fwd, without the workspace pair and without the optional
+ * entropy output (this variant returns logp and lse only).
  */
 #define DRK_NOALLOC_SCRATCH_BYTES (8u << 20)
 int drk_pg_logprob_fwd_noalloc(const void* hidden, const void* W, int32_t in_dtype, const int32_t* ids,

@@ -1,12 +1,12 @@
 """B200-native fused policy-gradient loss over the LM head (TRLOO + mismatch rejection sampling).
 
-`binding` wraps the C ABI of libdrk.so one to one; `synth` draws seeded synthetic inputs;
-`build` compiles the library.  Submodules are imported on first use so that `synth` can be used
-without the shared library.
+`binding` wraps the C ABI of libdrk.so one to one; `dp` strings the library calls together with the
+`torch.distributed` exchanges of the multi-GPU forms; `build` compiles the library.  Submodules are
+imported on first use.
 """
 import importlib
 
-__all__ = ["binding", "synth", "build"]
+__all__ = ["binding", "dp", "build"]
 
 
 def __getattr__(name):

@@ -8,6 +8,19 @@ namespace drk {
 
 thread_local int g_launches = 0;
 
+int sm_count() {
+  static int cached[64] = {};
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return 148; }
+  if (dev >= 0 && dev < 64 && cached[dev] > 0) return cached[dev];
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+    (void)cudaGetLastError();
+    return 148;
+  }
+  if (dev >= 0 && dev < 64) cached[dev] = n;
+  return n;
+}
+
 namespace {
 
 constexpr int kDefaultVChunk = 8192;
@@ -41,10 +54,10 @@ bool sizes_ok(int64_t T, int H, int V, int in_dtype) {
 
 // Chunk width for the tensor-core backward when the caller leaves it to the library: the multiple of
 // 256 that minimises the modelled time of the three per-chunk kernels.  Each kernel is persistent
-// over 148 SMs with 128x256 tiles, so its time is (waves of tiles) x (k-blocks per tile); a fixed
+// over the device's SMs with 128x256 tiles, so its time is (waves of tiles) x (k-blocks per tile); a fixed
 // cost per launch stands for fill and drain.  The dL buffer is kept below ~512 MiB (or 8192 columns).
 int auto_vchunk(int64_t T, int H, int V) {
-  const int64_t sms = 148, launch_cost = 96;
+  const int64_t sms = sm_count(), launch_cost = 96;
   const int64_t mt_T = ceil_div(T, 128), nt_H = ceil_div(H, 256), kb_H = ceil_div(H, 64), kb_T = ceil_div(T, 64);
   int64_t cap = ((int64_t)1 << 29) / (2 * (T > 0 ? T : 1)) / 256 * 256;
   if (cap < 8192) cap = 8192;

@@ -24,6 +24,10 @@ extern thread_local int g_launches;
     if (cudaGetLastError() != cudaSuccess) return DRK_ERR_CUDA; \
   } while (0)
 
+// Multiprocessors of the current device (148 on B200; the same number when no device can be queried, so that
+// size queries still answer on a host without a GPU).  Grids, wave models and split counts derive from it.
+int sm_count();
+
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 

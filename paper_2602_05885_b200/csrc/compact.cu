@@ -103,7 +103,7 @@ int launch_compact(const CompactArgs& a, cudaStream_t st) {
   DRK_LAUNCHED();
   rowmap_kernel<<<nblk, kBlk, 0, st>>>(a.coeff, a.T, a.blk_off, a.n_rows, map_len, a.rowmap);
   DRK_LAUNCHED();
-  gather_kernel<<<148 * 8, 256, 0, st>>>(a.hidden, a.H, a.rowmap, a.n_rows, a.hidden_c);
+  gather_kernel<<<sm_count() * 8, 256, 0, st>>>(a.hidden, a.H, a.rowmap, a.n_rows, a.hidden_c);
   DRK_LAUNCHED();
   return DRK_OK;
 }

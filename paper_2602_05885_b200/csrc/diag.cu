@@ -84,7 +84,8 @@ __global__ void diag_finalize_kernel(double* __restrict__ d) {
 
 static int launch_sumsq(const void* x, int dtype, size_t n, double* out, cudaStream_t st) {
   if (x == nullptr || n == 0) return DRK_OK;
-  const int blocks = (int)((n + 4095) / 4096 < 148 * 8 ? (n + 4095) / 4096 : 148 * 8);
+  const int64_t cap = (int64_t)sm_count() * 8;
+  const int blocks = (int)((n + 4095) / 4096 < cap ? (n + 4095) / 4096 : cap);
   if (dtype == DRK_BF16) sumsq_kernel<__nv_bfloat16><<<blocks, kDiagThreads, 0, st>>>((const __nv_bfloat16*)x, n, out);
   else sumsq_kernel<float><<<blocks, kDiagThreads, 0, st>>>((const float*)x, n, out);
   DRK_LAUNCHED();

@@ -321,7 +321,8 @@ __global__ void f32_to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16*
 
 int launch_f32_to_bf16(const float* src, __nv_bfloat16* dst, size_t n, cudaStream_t st) {
   if (n == 0) return DRK_OK;
-  const int blocks = (int)((n + 1023) / 1024 < 148 * 16 ? (n + 1023) / 1024 : 148 * 16);
+  const int64_t cap = (int64_t)sm_count() * 16;
+  const int blocks = (int)((n + 1023) / 1024 < cap ? (n + 1023) / 1024 : cap);
   f32_to_bf16_kernel<<<blocks, 256, 0, st>>>(src, dst, n);
   DRK_LAUNCHED();
   return DRK_OK;
@@ -340,7 +341,7 @@ int simt_nsplit(int64_t T, int V) {
   // enough blocks to fill the GPU a few times over, at least two 64-wide tiles per range
   const int64_t row_tiles = ceil_div(T, BM);
   const int ntiles = (V + BN - 1) / BN;
-  int64_t want = ceil_div(148 * 8, row_tiles > 0 ? row_tiles : 1);
+  int64_t want = ceil_div((int64_t)sm_count() * 8, row_tiles > 0 ? row_tiles : 1);
   if (want < 1) want = 1;
   if (want > ntiles) want = ntiles;
   if (want > 64) want = 64;

@@ -571,13 +571,6 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int sm_count() {
-  int dev = 0, n = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
-  return n;
-}
-
 template <int MODE, int CTAS>
 __global__ void umma_gemm_kernel(const __grid_constant__ CUtensorMap, const __grid_constant__ CUtensorMap,
                                  const UmmaParams);
@@ -666,7 +659,7 @@ int umma_nsplit(int64_t T, int V, int ctas, bool frugal) {
     if (ceil_div(n_tiles, per) > cap) per = ceil_div(n_tiles, cap);
     return (int)ceil_div(n_tiles, per);
   }
-  const int sms = 148 / ctas;
+  const int sms = sm_count() / ctas;
   double eff[33];
   double best_eff = -1.0;
   for (int ns = 1; ns <= 32; ++ns) {
@@ -712,7 +705,7 @@ int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st) {
   p.k_blocks = (int)ceil_div(a.H, TK);
   p.nj = a.nsplit;
   p.tiles_per_unit = (int)ceil_div(p.n_tiles, a.nsplit);
-  const int slots = 148 / ctas;
+  const int slots = sm_count() / ctas;
   if (a.nsplit > 32 || a.nsplit * 8 >= p.n_tiles) p.group_m = panel_group(TM * ctas, a.H);  // short units: panel budget
   else p.group_m = slots / a.nsplit > 0 ? slots / a.nsplit : 1;                    // long ranges: one wave
   p.rows = a.T; p.cols = a.V; p.v0 = 0; p.T = a.T;

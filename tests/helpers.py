@@ -13,7 +13,7 @@ import numpy as np
 import torch
 
 from oracle import drk_oracle as O
-from paper_2602_05885_b200 import synth
+from benchlib import synth
 
 # Tolerances (per-token log-prob, loss, gradients, advantages) as stated for the method's target.
 TOL_LOGP_BF16 = 2e-3
@@ -21,6 +21,14 @@ TOL_LOGP_F32 = 1e-4
 TOL_LOSS_REL = 1e-3
 TOL_GRAD_FRO = 1e-2
 TOL_ADV_REL = 1e-6
+# Rejection sampling (Sec. 5.1) compares a segment's MEAN log-ratio with thresholds only 1e-3 either side
+# of zero, so the decision is checked with a tolerance on that mean, not with the per-token one.  Both sides
+# read bit-identical inputs; the device's log-probs carry fp32 accumulation and ex2.approx rounding of
+# roughly 1e-5 per token, of either sign, and the mean over a segment's tokens is smaller still.  5e-5 is a
+# few times the largest deviation of ln(seg_w) from the oracle's mean seen on any case (each run reports it).
+TOL_MRS_MEAN = 5e-5
+# Largest admissible share of segments whose decision is within rounding of a threshold.
+MAX_AMBIGUOUS_FRAC = 0.10
 
 
 def f64(t: torch.Tensor) -> np.ndarray:
@@ -79,10 +87,45 @@ def oracle_advantages(rb: synth.RolloutBatch, gamma: float = 1.0):
     return G, A, N
 
 
+def nudge_into_band(logp: np.ndarray, rollout_logp: np.ndarray, mask: np.ndarray, cu: np.ndarray, seed: int,
+                    frac: float = 0.15, half_width: float = 6e-4) -> np.ndarray:
+    """Input recipe: moves a seeded 15 % of the clean samples inside the paper's acceptance band.
+
+    With i.i.d. per-token mismatch noise the mean log-ratio of a sample has a spread several times the band
+    ln 0.999 .. ln 1.001, so few samples (sometimes none) would be retained under the paper's constants.  For
+    the chosen samples (at least two; only samples without outlier tokens) a constant is added to the rollout
+    log-probs of their loss-masked tokens so that the mean log-ratio lands on a target spread evenly over
+    [-half_width, +half_width], i.e. at least 4e-4 away from either edge.  Returns float32 rollout log-probs;
+    everything downstream (oracle and device) sees only those."""
+    rl = np.asarray(rollout_logp, dtype=np.float64).copy()
+    S = len(cu) - 1
+    cands = []
+    for g in range(S):
+        sel = np.asarray(mask[cu[g]:cu[g + 1]]).astype(bool)
+        if sel.sum() >= 8:
+            d = (logp[cu[g]:cu[g + 1]] - rl[cu[g]:cu[g + 1]])[sel]
+            if np.abs(d).max() < 1.0:
+                cands.append(g)
+    if len(cands) < 4:
+        return rl.astype(np.float32)
+    rng = np.random.default_rng(seed)
+    n = max(2, int(round(frac * len(cands))))
+    chosen = rng.permutation(cands)[:n]
+    targets = rng.permutation(np.linspace(-half_width, half_width, n))
+    for g, target in zip(chosen, targets):
+        a, b = int(cu[g]), int(cu[g + 1])
+        sel = np.asarray(mask[a:b]).astype(bool)
+        d = (logp[a:b] - rl[a:b])[sel]
+        shift = float(d.mean()) - float(target)      # delta = logp - rollout: raise the rollout side by the excess
+        seg = rl[a:b]
+        seg[sel] += shift
+    return rl.astype(np.float32)
+
+
 def build_case(name: str, *, H: int, V: int, dtype: torch.dtype, P: int, K: int, Tmax: int,
                len_lo: int, len_hi: int, capacity: int, seed: int, sigma: float = 0.05,
                ragged: bool = False, ctx_frac: float = 0.0, outlier_frac: float = 0.0,
-               lead_pad: int = 0, microbatch: int = 0, uniform_ids: bool = False) -> Case:
+               lead_pad: int = 0, microbatch: int = 0, uniform_ids: bool = False, nudge: bool = True) -> Case:
     rb = synth.rollout_batch(P, K, Tmax, len_lo, len_hi, seed, ragged=ragged, ctx_frac=ctx_frac)
     plans = synth.pack_first_fit(rb, capacity - lead_pad)
     plan = plans[microbatch]
@@ -100,7 +143,10 @@ def build_case(name: str, *, H: int, V: int, dtype: torch.dtype, P: int, K: int,
     else:
         ids = sample_ids_from_policy(s, u.numpy())
     logp, lse = O.token_logprob(s, ids)
-    rollout_logp = torch.from_numpy((logp + noise.numpy().astype(np.float64)).astype(np.float32))
+    rl = (logp + noise.numpy().astype(np.float64)).astype(np.float32)
+    if nudge:
+        rl = nudge_into_band(logp, rl, mask.numpy(), cu.numpy(), seed + 5)
+    rollout_logp = torch.from_numpy(rl)
     _, A, _ = oracle_advantages(rb)
     seg_adv = torch.from_numpy(A[seg_rollout.numpy(), seg_turn.numpy()].astype(np.float32))
     return Case(name, dtype, hidden, W, torch.from_numpy(ids.astype(np.int32)), rollout_logp, mask, cu,
@@ -130,12 +176,16 @@ def build_plain_case(name: str, *, T: int, H: int, V: int, dtype: torch.dtype, S
 # Oracle evaluation of a case under given MRS parameters
 # ---------------------------------------------------------------------------
 
-def wide_band(case: Case):
-    """(lo, hi) = exp(-+q) with q the oracle's median |mean delta|: about half the samples pass."""
-    m = O.mrs(case.logp, f64(case.rollout_logp), case.loss_mask.numpy(), case.cu.numpy(), lo=0.0, hi=math.inf)
-    nz = m.n_masked > 0
-    q = float(np.median(np.abs(m.mean_delta[nz]))) if nz.any() else 1e-3
+def band_from_means(mean_delta: np.ndarray):
+    """(lo, hi) = exp(-+q) as float32, q midway between two adjacent order statistics of |mean delta| next to
+    the median: about half the samples pass and none sits on a threshold by construction."""
+    q = synth.threshold_between(np.abs(mean_delta))
     return float(np.float32(math.exp(-q))), float(np.float32(math.exp(q)))
+
+
+def wide_band(case: Case):
+    m = O.mrs(case.logp, f64(case.rollout_logp), case.loss_mask.numpy(), case.cu.numpy(), lo=0.0, hi=math.inf)
+    return band_from_means(m.mean_delta[m.n_masked > 0])
 
 
 def oracle_eval(case: Case, lo: float, hi: float, veto: float, norm: int = 0, explicit_scale: float = 1.0,
@@ -170,8 +220,52 @@ def rel_fro(a: np.ndarray, b: np.ndarray) -> float:
     return float(np.linalg.norm(a - b)) / nb
 
 
+_report_lines = []
+
+
+def report(line: str):
+    """Parity figures worth keeping (tolerance headroom, ambiguous counts): printed, and appended to the file
+    named by DRK_PARITY_REPORT when set."""
+    import os
+    print(line)
+    path = os.environ.get("DRK_PARITY_REPORT")
+    if path:
+        with open(path, "a") as f:
+            f.write(line + "\n")
+
+
+def check_decisions(name: str, m: O.MrsResult, seg_w_dev: np.ndarray, keep_dev: np.ndarray, lo: float, hi: float,
+                    veto: float, tol_tok: float, paper_decisive: bool = False, caller_keep=None):
+    """The rejection decision of every segment against the oracle's.
+
+    ln(seg_w) must match the oracle's mean log-ratio within TOL_MRS_MEAN.  A segment is ambiguous only if its
+    mean lies within TOL_MRS_MEAN of a band edge or its smallest log-ratio within the per-token tolerance of
+    the veto threshold; all other decisions must be identical, and few segments may be ambiguous.  With
+    paper_decisive the case must also hold two unambiguous retained and two unambiguous rejected samples.
+    Returns the mask of ambiguous segments."""
+    nz = m.n_masked > 0
+    seg_w_dev = np.asarray(seg_w_dev, dtype=np.float64)
+    assert (seg_w_dev[~nz] == 1.0).all()
+    mean_err = np.abs(np.log(seg_w_dev[nz]) - m.mean_delta[nz]).max(initial=0.0)
+    assert mean_err <= TOL_MRS_MEAN, f"{name}: ln(seg_w) deviates from the oracle's mean log-ratio by {mean_err}"
+    amb = ambiguous_segments(m, lo, hi, veto, tol_mean=TOL_MRS_MEAN, tol_tok=tol_tok)
+    expect = m.keep if caller_keep is None else caller_keep
+    mismatch = (np.asarray(keep_dev).astype(bool) != expect) & ~amb
+    assert not mismatch.any(), f"{name}: keep differs on unambiguous segments {np.nonzero(mismatch)[0]}"
+    S = len(m.keep)
+    assert amb.sum() <= max(1, int(MAX_AMBIGUOUS_FRAC * S)), f"{name}: {amb.sum()} of {S} segments ambiguous"
+    kept_clear = int((m.keep & ~amb).sum())
+    rej_clear = int((~m.keep & nz & ~amb).sum())
+    if paper_decisive:
+        assert kept_clear >= 2 and rej_clear >= 2, f"{name}: {kept_clear} retained / {rej_clear} rejected decisive"
+    report(f"mrs {name} band=[{lo:.6f},{hi:.6f}] veto={veto:g}: segments={S} ambiguous={int(amb.sum())} "
+           f"retained={kept_clear} rejected={rej_clear} max|ln seg_w - mean|={mean_err:.2e}")
+    return amb
+
+
 def check_against_oracle(case: Case, dev: Dict, lo: float, hi: float, veto: float, norm: int = 0,
-                         explicit_scale: float = 1.0, seg_adv=None, dW_before: Optional[np.ndarray] = None):
+                         explicit_scale: float = 1.0, seg_adv=None, dW_before: Optional[np.ndarray] = None,
+                         paper_decisive: bool = False):
     """dev: dict of CPU tensors from the device path (logp, lse, seg_w, seg_keep, loss, counters, dH, dW)."""
     tol_logp = TOL_LOGP_F32 if case.dtype == torch.float32 else TOL_LOGP_BF16
     T, S = case.T, case.S
@@ -186,15 +280,9 @@ def check_against_oracle(case: Case, dev: Dict, lo: float, hi: float, veto: floa
     first = oracle_eval(case, lo, hi, veto, norm, explicit_scale, seg_adv=seg_adv, want_grads=False)
     m = first["mrs"]
     keep_dev = dev["seg_keep"].numpy().astype(bool)
-    amb = ambiguous_segments(m, lo, hi, veto, tol_mean=tol_logp, tol_tok=tol_logp)
-    mismatch = (keep_dev != m.keep) & ~amb
-    assert not mismatch.any(), f"keep differs on unambiguous segments {np.nonzero(mismatch)[0]}"
+    amb = check_decisions(case.name, m, f64(dev["seg_w"]), keep_dev, lo, hi, veto, tol_logp, paper_decisive)
+    # gradients and loss follow the device's flags on the (few) ambiguous segments, the oracle's elsewhere
     ref = oracle_eval(case, lo, hi, veto, norm, explicit_scale, keep_override=keep_dev, seg_adv=seg_adv)
-    if S > 0:
-        nz = m.n_masked > 0
-        werr = np.abs(f64(dev["seg_w"]) - m.w)[nz] / m.w[nz]
-        assert werr.max(initial=0.0) <= 2 * tol_logp, f"seg_w rel err {werr.max()}"
-        assert (f64(dev["seg_w"])[~nz] == 1.0).all()
     counters = dev["counters"].numpy()
     assert counters[0] == ref["kept_tokens"] and counters[1] == ref["masked_tokens"]
     assert counters[2] == ref["kept_segs"]

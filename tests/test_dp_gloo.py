@@ -10,7 +10,8 @@ import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
 
-from paper_2602_05885_b200 import dp, synth
+from paper_2602_05885_b200 import dp
+from benchlib import synth
 
 
 def _free_port():

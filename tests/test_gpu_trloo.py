@@ -5,7 +5,7 @@ import torch
 
 from oracle import drk_oracle as O
 from paper_2602_05885_b200 import binding as B
-from paper_2602_05885_b200 import synth
+from benchlib import synth
 from tests.helpers import TOL_ADV_REL
 
 pytestmark = pytest.mark.gpu

@@ -1,7 +1,7 @@
 """The seeded input generators: determinism and structural validity."""
 import torch
 
-from paper_2602_05885_b200 import synth
+from benchlib import synth
 
 
 def test_rollout_batch_is_deterministic_and_well_formed():

@@ -11,7 +11,7 @@ import pytest
 import torch
 
 from paper_2602_05885_b200 import binding as B
-from paper_2602_05885_b200 import synth
+from benchlib import synth
 from tests.helpers import TOL_LOGP_BF16, TOL_LOGP_F32
 
 pytestmark = pytest.mark.gpu
@@ -38,20 +38,24 @@ def _both(hidden, W, ids, engine=B.DRK_ENGINE_AUTO):
     return (logp.cpu(), lse.cpu(), int(status.item())), (ref_logp.cpu(), ref_lse.cpu(), int(ref_status.item()))
 
 
+@pytest.mark.parametrize("engine", [B.DRK_ENGINE_AUTO, B.DRK_ENGINE_UMMA_1CTA, B.DRK_ENGINE_SIMT],
+                         ids=["pairs", "single-cta", "ffma"])
 @pytest.mark.parametrize("dtype,tol", [(torch.bfloat16, TOL_LOGP_BF16), (torch.float32, TOL_LOGP_F32)])
-def test_two_calls_in_a_row_match_the_workspace_entry_point(dtype, tol):
+def test_two_calls_in_a_row_match_the_workspace_entry_point(dtype, tol, engine):
+    # every route into the fixed array: CTA pairs, one CTA per tile, and the FFMA kernels (which fp32 inputs
+    # always take, whatever the engine says)
     dev = torch.device("cuda:0")
     # first call: larger problem, with two invalid ids so that stale target logits would show up later
     h1, W1, ids1 = _inputs(700, 512, 9000, dtype, 21, dev)
     ids1[3] = -1
     ids1[650] = 9000
-    got, ref = _both(h1, W1, ids1)
+    got, ref = _both(h1, W1, ids1, engine)
     assert got[2] == ref[2] and (got[2] & B.DRK_STATUS_BAD_ID)
     assert (got[0] - ref[0]).abs().max() <= tol and (got[1] - ref[1]).abs().max() <= tol
     # second call, different sizes and data, right after the first
     h2, W2, ids2 = _inputs(333, 256, 4100, dtype, 22, dev)
     ids2[3] = 4100                                   # invalid again: its target must read as 0, not as a leftover
-    got, ref = _both(h2, W2, ids2)
+    got, ref = _both(h2, W2, ids2, engine)
     assert got[2] == ref[2]
     assert (got[0] - ref[0]).abs().max() <= tol and (got[1] - ref[1]).abs().max() <= tol
     assert abs(float(got[0][3]) + float(got[1][3])) < 1e-6
