@@ -13,9 +13,18 @@
  *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*, NULL =
  *     the legacy default stream) and return without synchronising.  Scalar
  *     results (loss, counters, status) stay in device memory.
- *   - Return value: DRK_OK or a negative drk_status.  On a negative return
- *     nothing was enqueued.  Conditions only the device can see set bits in the
- *     device word `*status` (DRK_STATUS_*); no kernel traps or spins unbounded.
+ *   - Return value: DRK_OK or a negative drk_status.  Arguments, sizes, the
+ *     device's architecture, kernel attributes and every tensor map are checked
+ *     or built on the host before the first enqueue: on DRK_ERR_INVALID_ARG,
+ *     _UNSUPPORTED, _WORKSPACE or _ARCH nothing was enqueued, and DRK_ERR_CUDA
+ *     from those host steps enqueues nothing either.  The one exception is
+ *     DRK_ERR_CUDA raised by an enqueue itself (the runtime refusing a launch,
+ *     a memset or an event record part-way through a call): earlier kernels of
+ *     that call are then already on the stream and the outputs are undefined.
+ *     Conditions only the device can see set bits in the device word `*status`
+ *     (DRK_STATUS_*); no kernel traps or spins unbounded.
+ *   - Sizes that depend on the device (workspace bytes, chunk widths) are
+ *     computed for the current device's multiprocessor count.
  *   - All matrices are row-major and dense (leading dimension = row length).
  *   - Row t of `hidden` predicts the token `ids[t]`; the caller has already
  *     applied the next-token shift.
@@ -338,6 +347,13 @@ int drk_selftest_bounded_wait(uint32_t limit_ms, uint32_t* status, uint64_t* wai
 
 /* Number of kernels the last call on this host thread enqueued (0 after an error). */
 int drk_last_launch_count(void);
+
+/*
+ * Number of TMA tensor maps this process has encoded so far (no counterpart in the paper).  Maps depend on a
+ * buffer's address and geometry only and are cached, so a call that repeats an earlier call's pointers and
+ * sizes (the steady state of a training loop) adds nothing to this count.
+ */
+uint64_t drk_tensor_map_encodes(void);
 
 const char* drk_status_string(int status);
 int drk_version(void);

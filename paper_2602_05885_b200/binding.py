@@ -135,6 +135,8 @@ def load() -> ctypes.CDLL:
     lib.drk_selftest_bounded_wait.restype = ctypes.c_int
     lib.drk_last_launch_count.argtypes = []
     lib.drk_last_launch_count.restype = ctypes.c_int
+    lib.drk_tensor_map_encodes.argtypes = []
+    lib.drk_tensor_map_encodes.restype = ctypes.c_uint64
     lib.drk_status_string.argtypes = [ctypes.c_int]
     lib.drk_status_string.restype = ctypes.c_char_p
     lib.drk_version.argtypes = []
@@ -180,6 +182,10 @@ def drk_version() -> int:
 
 def drk_last_launch_count() -> int:
     return load().drk_last_launch_count()
+
+
+def drk_tensor_map_encodes() -> int:
+    return int(load().drk_tensor_map_encodes())
 
 
 def drk_pg_params_default() -> drk_pg_params:

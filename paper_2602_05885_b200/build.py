@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_PATH = os.path.join(HERE, "libdrk.so")
 SOURCES = ["api.cu", "trloo.cu", "mrs.cu", "simt.cu", "umma_kernels.cu", "noalloc.cu", "compact.cu", "reward.cu", "diag.cu"]
-HEADERS = ["common.cuh", "umma.cuh", os.path.join("..", "..", "include", "drk.h")]
+HEADERS = ["common.cuh", "umma.cuh", "umma_plan.cuh", os.path.join("..", "..", "include", "drk.h")]
 
 
 def _nvcc() -> str:

@@ -1,5 +1,6 @@
 // C-ABI entry points of libdrk.so: argument validation, workspace carving, dispatch.
 #include "common.cuh"
+#include "umma_plan.cuh"
 #include <cmath>
 #include <limits>
 #include <nvtx3/nvToolsExt.h>   // header-only; ranges cost nothing unless a profiler is attached
@@ -161,6 +162,16 @@ bool params_ok(const drk_pg_params& p) {
   return true;
 }
 
+UmmaFwdArgs umma_fwd_args(const void* hidden, const void* W, const int32_t* ids, int64_t T, int H, int V, int engine,
+                          const FwdWs& w, float* logp, float* lse, float* entropy, uint32_t* status,
+                          const __nv_bfloat16* hidden_c, const int32_t* rowmap, const int32_t* n_rows, int id_off,
+                          float* stats) {
+  UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, w.part, w.tgt, w.nsplit, status, umma_ctas(engine), entropy,
+                hidden_c, rowmap, n_rows};
+  a.id_off = id_off; a.stats = stats;
+  return a;
+}
+
 int run_fwd(const void* hidden, const void* W, int in_dtype, const int32_t* ids, int64_t T, int H, int V,
             bool simt, int engine, const FwdWs& w, float* logp, float* lse, float* entropy, uint32_t* status,
             cudaStream_t st, const __nv_bfloat16* hidden_c = nullptr, const int32_t* rowmap = nullptr,
@@ -170,10 +181,12 @@ int run_fwd(const void* hidden, const void* W, int in_dtype, const int32_t* ids,
     a.id_off = id_off; a.stats = stats;
     return launch_simt_fwd(a, st);
   }
-  UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, w.part, w.tgt, w.nsplit, status, umma_ctas(engine), entropy,
-                hidden_c, rowmap, n_rows};
-  a.id_off = id_off; a.stats = stats;
-  return launch_umma_fwd(a, st);
+  // plan (host only: kernel attributes, tensor maps) first, then enqueue
+  UmmaFwdPlan plan;
+  int rc = plan_umma_fwd(umma_fwd_args(hidden, W, ids, T, H, V, engine, w, logp, lse, entropy, status, hidden_c, rowmap,
+                                       n_rows, id_off, stats), &plan);
+  if (rc != DRK_OK) return rc;
+  return enqueue_umma_fwd(plan, st);
 }
 
 // Vocabulary-range mode of the fused call: log-probs come from all ranges' statistics instead of a forward
@@ -228,6 +241,27 @@ int loss_fwd_bwd_impl(const void* hidden, const void* W, int32_t in_dtype, const
 
   auto fail = [&](int code) { g_launches = 0; return code; };
 
+  // Tensor-core path: every host step that can fail (driver entry point, kernel attributes, all tensor maps
+  // of the forward and of every vocabulary chunk of the backward) runs here, before the first enqueue.
+  const bool fwd_here = T > 0 && sh == nullptr && p.reuse_forward == 0;
+  const bool fwd_rows = fwd_here && p.forward_rows == 1 && !simt;
+  UmmaFwdPlan fplan;
+  UmmaBwdPlan bplan;
+  if (!simt && T > 0) {
+    if (fwd_here) {
+      rc = plan_umma_fwd(umma_fwd_args(hidden, W, ids, T, H, V, p.engine, fw, logp, lse, entropy, status,
+                                       fwd_rows ? bw.hidden_c : nullptr, fwd_rows ? bw.rowmap : nullptr,
+                                       fwd_rows ? bw.n_rows : nullptr, 0, nullptr), &fplan);
+      if (rc != DRK_OK) return fail(rc);
+    }
+    UmmaBwdArgs b{hidden, W, ids, T, H, V, lse, bw.coeff, static_cast<__nv_bfloat16*>(bw.dL), bw.vc,
+                  dH, p.dh_dtype, bw.dH_acc, dW, p.dw_dtype, p.dw_accumulate, status, umma_ctas(p.engine),
+                  bw.hidden_c, bw.rowmap, bw.n_rows, p.dw_chunk_events};
+    b.id_off = id_off;
+    rc = plan_umma_bwd(b, &bplan);
+    if (rc != DRK_OK) return fail(rc);
+  }
+
   Range call_range(sh ? "drk_pg_shard_loss_bwd" : "drk_pg_loss_fwd_bwd");
   if (T > 0 && sh == nullptr && p.reuse_forward == 1) {
     // logp and lse come from an earlier forward over the same operands
@@ -248,12 +282,12 @@ int loss_fwd_bwd_impl(const void* hidden, const void* W, int32_t in_dtype, const
         cudaMemsetAsync(lse, 0, sizeof(float) * (size_t)T, st) != cudaSuccess ||
         (entropy && cudaMemsetAsync(entropy, 0, sizeof(float) * (size_t)T, st) != cudaSuccess))
       return fail(DRK_ERR_CUDA);
-    rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, p.engine, fw, logp, lse, entropy, status, st, bw.hidden_c,
-                 bw.rowmap, bw.n_rows);
+    rc = enqueue_umma_fwd(fplan, st);
     if (rc != DRK_OK) return fail(rc);
   } else if (T > 0) {
     Range r("drk: forward");
-    rc = run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, p.engine, fw, logp, lse, entropy, status, st);
+    rc = simt ? run_fwd(hidden, W, in_dtype, ids, T, H, V, simt, p.engine, fw, logp, lse, entropy, status, st)
+              : enqueue_umma_fwd(fplan, st);
     if (rc != DRK_OK) return fail(rc);
   }
   {
@@ -290,11 +324,7 @@ int loss_fwd_bwd_impl(const void* hidden, const void* W, int32_t in_dtype, const
                    bw.rowmap, bw.hidden_c};
     rc = launch_compact(ca, st);
     if (rc != DRK_OK) return fail(rc);
-    UmmaBwdArgs b{hidden, W, ids, T, H, V, lse, bw.coeff, static_cast<__nv_bfloat16*>(bw.dL), bw.vc,
-                  dH, p.dh_dtype, bw.dH_acc, dW, p.dw_dtype, p.dw_accumulate, status, umma_ctas(p.engine),
-                  bw.hidden_c, bw.rowmap, bw.n_rows, p.dw_chunk_events};
-    b.id_off = id_off;
-    rc = launch_umma_bwd(b, st);
+    rc = enqueue_umma_bwd(bplan, st);
   }
   if (rc != DRK_OK) return fail(rc);
   return DRK_OK;
@@ -480,6 +510,8 @@ int drk_selftest_bounded_wait(uint32_t limit_ms, uint32_t* status, uint64_t* wai
 }
 
 int drk_last_launch_count(void) { return g_launches; }
+
+uint64_t drk_tensor_map_encodes(void) { return umma_map_encodes(); }
 
 const char* drk_status_string(int s) {
   switch (s) {

@@ -19,6 +19,7 @@
 //     capture.
 // No cudaMalloc, cudaFree or allocating library routine is called.
 #include "common.cuh"
+#include "umma_plan.cuh"
 #include <mutex>
 
 namespace drk {
@@ -89,14 +90,19 @@ extern "C" int drk_pg_logprob_fwd_noalloc(const void* hidden, const void* W, int
   float* part = reinterpret_cast<float*>(base);
   float* tgt = reinterpret_cast<float*>(static_cast<char*>(base) + part_bytes);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  UmmaFwdPlan plan;
+  if (!simt) {   // kernel attributes and tensor maps (host only) before anything is enqueued
+    UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, part, tgt, nsplit, status, ctas, nullptr, nullptr, nullptr, nullptr};
+    rc = plan_umma_fwd(a, &plan);
+    if (rc != DRK_OK) return rc;
+  }
   if (cudaMemsetAsync(tgt, 0, tgt_bytes, st) != cudaSuccess) return DRK_ERR_CUDA;
 
   if (simt) {
     SimtFwdArgs a{hidden, W, in_dtype, ids, T, H, V, logp, lse, part, tgt, nsplit, status, nullptr};
     rc = launch_simt_fwd(a, st);
   } else {
-    UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, part, tgt, nsplit, status, ctas, nullptr, nullptr, nullptr, nullptr};
-    rc = launch_umma_fwd(a, st);
+    rc = enqueue_umma_fwd(plan, st);
   }
   if (rc != DRK_OK) g_launches = 0;
   return rc;

@@ -20,7 +20,8 @@
 // in-flight copies and MMAs, frees tensor memory and returns.
 #include "common.cuh"
 #include "umma.cuh"
-#include <cuda.h>
+#include "umma_plan.cuh"
+#include <atomic>
 #include <math_constants.h>
 #include <mutex>
 
@@ -556,26 +557,75 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// Row-major bf16 matrix [outer, inner] with row pitch `pitch_elems`; box = box_inner x box_outer,
-// 128-byte swizzle, zero fill outside the extents.
-bool make_map(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, uint64_t pitch_elems,
-              uint32_t box_inner, uint32_t box_outer) {
+// Tensor maps depend on the address and geometry only, never on the contents, so a map encoded once serves
+// every later call on the same buffer: a steady-state training step (same W, hidden and workspace pointers)
+// encodes nothing.  Small direct-mapped table with four probes, shared by all threads.
+struct MapKey {
+  const void* base; uint64_t inner, outer, pitch_bytes; uint32_t box_inner, box_outer, dtype;
+  bool operator==(const MapKey& o) const {
+    return base == o.base && inner == o.inner && outer == o.outer && pitch_bytes == o.pitch_bytes &&
+           box_inner == o.box_inner && box_outer == o.box_outer && dtype == o.dtype;
+  }
+};
+struct MapEntry { MapKey key; CUtensorMap map; bool used; };
+constexpr int kMapTable = 512;
+std::mutex g_map_mu;
+MapEntry g_map_table[kMapTable] = {};
+std::atomic<uint64_t> g_map_encodes{0};
+
+size_t map_hash(const MapKey& k) {
+  uint64_t h = reinterpret_cast<uintptr_t>(k.base) * 0x9E3779B97F4A7C15ull;
+  h ^= (k.inner + 0x632BE59BD9B4E019ull) * 0xFF51AFD7ED558CCDull;
+  h ^= (k.outer + (h >> 29)) * 0xC4CEB9FE1A85EC53ull;
+  h ^= ((uint64_t)k.box_inner << 40) ^ ((uint64_t)k.box_outer << 20) ^ k.dtype ^ (k.pitch_bytes * 0x2545F4914F6CDD1Dull);
+  return (size_t)((h ^ (h >> 32)) % kMapTable);
+}
+
+// Row-major matrix [outer, inner] of 2-byte (bf16) or 4-byte (fp32) elements with row pitch `pitch_elems`;
+// box = box_inner x box_outer, 128-byte swizzle, zero fill outside the extents on loads (stores are clipped).
+bool make_map_typed(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, uint64_t pitch_elems,
+                    uint32_t box_inner, uint32_t box_outer, bool f32) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
+  const uint32_t esz = f32 ? 4 : 2;
+  const MapKey key{base, inner, outer, pitch_elems * esz, box_inner, box_outer, f32 ? 1u : 0u};
+  const size_t h = map_hash(key);
+  {
+    std::lock_guard<std::mutex> lock(g_map_mu);
+    for (int i = 0; i < 4; ++i) {
+      const MapEntry& e = g_map_table[(h + i) % kMapTable];
+      if (e.used && e.key == key) { *m = e.map; return true; }
+    }
+  }
   cuuint64_t dims[2] = {inner, outer};
-  cuuint64_t strides[1] = {pitch_elems * 2};
+  cuuint64_t strides[1] = {pitch_elems * esz};
   cuuint32_t box[2] = {box_inner, box_outer};
   cuuint32_t estr[2] = {1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  if (fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
+         strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return false;
+  g_map_encodes.fetch_add(1, std::memory_order_relaxed);
+  std::lock_guard<std::mutex> lock(g_map_mu);
+  int slot = (int)h;
+  for (int i = 0; i < 4; ++i)
+    if (!g_map_table[(h + i) % kMapTable].used) { slot = (int)((h + i) % kMapTable); break; }
+  g_map_table[slot].key = key;
+  g_map_table[slot].map = *m;
+  g_map_table[slot].used = true;
+  return true;
+}
+
+bool make_map(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, uint64_t pitch_elems,
+              uint32_t box_inner, uint32_t box_outer) {
+  return make_map_typed(m, base, inner, outer, pitch_elems, box_inner, box_outer, false);
 }
 
 template <int MODE, int CTAS>
 __global__ void umma_gemm_kernel(const __grid_constant__ CUtensorMap, const __grid_constant__ CUtensorMap,
                                  const UmmaParams);
 
-// How many two-CTA clusters of this kernel the device can hold at once (one CTA per SM).
+// How many two-CTA clusters of this kernel the device can hold at once (one CTA per SM); 0 if the query fails.
 int resident_pairs() {
   static int cached[64] = {};
   int dev = 0;
@@ -594,8 +644,7 @@ int resident_pairs() {
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
-      cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) {
+  if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) {
     (void)cudaGetLastError();
     n = sm_count() / 2;
   }
@@ -605,11 +654,39 @@ int resident_pairs() {
 }
 
 template <int MODE, int CTAS>
+bool set_smem_attr() {
+  if (cudaFuncSetAttribute(umma_gemm_kernel<MODE, CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) !=
+      cudaSuccess) {
+    (void)cudaGetLastError();
+    return false;
+  }
+  return true;
+}
+
+// Everything on the host that can fail and does not depend on the call's arguments: the driver entry point
+// for tensor-map encoding, the shared-memory attribute of all eight kernel instantiations, and the
+// residency query.  Done once per device; later calls return the cached answer.
+int umma_prepare() {
+  static std::mutex mu;
+  static int state[64] = {};   // 0 unknown, 1 ready, -1 failed
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DRK_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(mu);
+  if (state[dev] == 0) {
+    bool ok = get_encode_fn() != nullptr;
+    ok = ok && set_smem_attr<FWD, 1>() && set_smem_attr<DL, 1>() && set_smem_attr<DW, 1>() && set_smem_attr<DH, 1>();
+    ok = ok && set_smem_attr<FWD, 2>() && set_smem_attr<DL, 2>() && set_smem_attr<DW, 2>() && set_smem_attr<DH, 2>();
+    if (ok) (void)resident_pairs();
+    state[dev] = ok ? 1 : -1;
+  }
+  return state[dev] == 1 ? DRK_OK : DRK_ERR_CUDA;
+}
+
+template <int MODE, int CTAS>
 int launch_mode_ctas(const CUtensorMap& a, const CUtensorMap& b, UmmaParams p, cudaStream_t st) {
   p.num_units = p.m_tiles * p.nj;   // upper bound when the row count lives on the device
   if (p.num_units <= 0) return DRK_OK;
   auto kern = umma_gemm_kernel<MODE, CTAS>;
-  DRK_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(NUM_THREADS);
   cfg.dynamicSmemBytes = SMEM_BYTES;
@@ -638,6 +715,8 @@ int launch_mode(int ctas, const CUtensorMap& a, const CUtensorMap& b, const Umma
 }
 
 }  // namespace
+
+uint64_t umma_map_encodes() { return g_map_encodes.load(std::memory_order_relaxed); }
 
 // Number of vocabulary ranges per row tile in the forward (each work unit = one row tile x one range,
 // with its own partial max / sum-exp per row).
@@ -691,14 +770,24 @@ int launch_bounded_wait_selftest(uint32_t limit_ms, uint32_t* status, uint64_t* 
   return DRK_OK;
 }
 
-int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st) {
+// ---- forward ----------------------------------------------------------------------------------------------
+
+int plan_umma_fwd(const UmmaFwdArgs& a, UmmaFwdPlan* plan) {
+  int rc = umma_prepare();
+  if (rc != DRK_OK) return rc;
+  plan->a = a;
   const int ctas = a.ctas == 2 ? 2 : 1;
-  CUtensorMap mh, mw;
   // With a row map the forward runs over the gathered rows (hidden_c) only; the kernels read their number.
   const void* hid = a.rowmap ? (const void*)a.hidden_c : a.hidden;
   const int64_t hid_rows = a.rowmap ? ceil_div(a.T, 256) * 256 : a.T;
-  if (!make_map(&mh, hid, a.H, hid_rows, a.H, TK, TM)) return DRK_ERR_CUDA;
-  if (!make_map(&mw, a.W, a.H, a.V, a.H, TK, TN / ctas)) return DRK_ERR_CUDA;
+  if (!make_map(&plan->mh, hid, a.H, hid_rows, a.H, TK, TM)) return DRK_ERR_CUDA;
+  if (!make_map(&plan->mw, a.W, a.H, a.V, a.H, TK, TN / ctas)) return DRK_ERR_CUDA;
+  return DRK_OK;
+}
+
+int enqueue_umma_fwd(const UmmaFwdPlan& plan, cudaStream_t st) {
+  const UmmaFwdArgs& a = plan.a;
+  const int ctas = a.ctas == 2 ? 2 : 1;
   UmmaParams p{};
   p.m_tiles = (int)ceil_div(a.T, TM * ctas);
   p.n_tiles = (int)ceil_div(a.V, TN);
@@ -713,7 +802,7 @@ int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st) {
   p.ids = a.ids; p.part = a.part; p.tgt = a.tgt; p.status = a.status;
   p.want_entropy = a.entropy != nullptr || a.stats != nullptr;   // the statistics carry the same third sum
   p.rowmap = a.rowmap; p.n_rows = a.n_rows;
-  int rc = launch_mode<FWD>(ctas, mh, mw, p, st);
+  int rc = launch_mode<FWD>(ctas, plan.mh, plan.mw, p, st);
   if (rc != DRK_OK) return rc;
   if (a.stats != nullptr)
     return launch_shard_stats(a.part, a.tgt, a.ids, a.id_off, a.T, a.V, a.nsplit, a.stats, a.status, st);
@@ -721,17 +810,43 @@ int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st) {
                           a.n_rows, st);
 }
 
-int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {
+int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st) {
+  UmmaFwdPlan plan;
+  int rc = plan_umma_fwd(a, &plan);
+  if (rc != DRK_OK) return rc;
+  return enqueue_umma_fwd(plan, st);
+}
+
+// ---- backward ---------------------------------------------------------------------------------------------
+
+int plan_umma_bwd(const UmmaBwdArgs& a, UmmaBwdPlan* plan) {
+  int rc = umma_prepare();
+  if (rc != DRK_OK) return rc;
+  plan->a = a;
   const int ctas = a.ctas == 2 ? 2 : 1;
-  const int TMC = TM * ctas;   // rows of one work unit's tile
   // The row dimension of the three contractions runs over the compacted rows (hidden_c, rowmap);
   // buffers are sized for the worst case (every row kept), the kernels read the actual count.
   const int64_t rows_cap = ceil_div(a.T, 256) * 256;
-  CUtensorMap mh_k, mw_k, mh_mn, mw_mn;
-  if (!make_map(&mh_k, a.hidden_c, a.H, rows_cap, a.H, TK, TM)) return DRK_ERR_CUDA;
-  if (!make_map(&mw_k, a.W, a.H, a.V, a.H, TK, TN / ctas)) return DRK_ERR_CUDA;
-  if (!make_map(&mh_mn, a.hidden_c, a.H, rows_cap, a.H, 64, TK)) return DRK_ERR_CUDA;
-  if (!make_map(&mw_mn, a.W, a.H, a.V, a.H, 64, TK)) return DRK_ERR_CUDA;
+  if (!make_map(&plan->mh_k, a.hidden_c, a.H, rows_cap, a.H, TK, TM)) return DRK_ERR_CUDA;
+  if (!make_map(&plan->mw_k, a.W, a.H, a.V, a.H, TK, TN / ctas)) return DRK_ERR_CUDA;
+  if (!make_map(&plan->mh_mn, a.hidden_c, a.H, rows_cap, a.H, 64, TK)) return DRK_ERR_CUDA;
+  if (!make_map(&plan->mw_mn, a.W, a.H, a.V, a.H, 64, TK)) return DRK_ERR_CUDA;
+  const int n_chunks = (int)ceil_div(a.V, a.vc);
+  plan->mdl_k.resize(n_chunks);
+  plan->mdl_mn.resize(n_chunks);
+  for (int c = 0; c < n_chunks; ++c) {
+    const int v0 = c * a.vc;
+    const int vc_this = a.V - v0 < a.vc ? a.V - v0 : a.vc;
+    if (!make_map(&plan->mdl_k[c], a.dL, vc_this, rows_cap, a.vc, TK, TM)) return DRK_ERR_CUDA;
+    if (!make_map(&plan->mdl_mn[c], a.dL, vc_this, rows_cap, a.vc, 64, TK)) return DRK_ERR_CUDA;
+  }
+  return DRK_OK;
+}
+
+int enqueue_umma_bwd(const UmmaBwdPlan& plan, cudaStream_t st) {
+  const UmmaBwdArgs& a = plan.a;
+  const int ctas = a.ctas == 2 ? 2 : 1;
+  const int TMC = TM * ctas;   // rows of one work unit's tile
   float* dh_acc = (a.dh_dtype == DRK_F32) ? (float*)a.dH : a.dH_acc;
   // rows that are not in the compacted set keep this zero
   DRK_CUDA_CHECK(cudaMemsetAsync(a.dH, 0, (size_t)a.T * a.H * (a.dh_dtype == DRK_BF16 ? 2 : 4), st));
@@ -739,9 +854,8 @@ int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {
   int chunk = 0;
   for (int v0 = 0; v0 < a.V; v0 += a.vc, ++chunk) {
     const int vc_this = a.V - v0 < a.vc ? a.V - v0 : a.vc;
-    CUtensorMap mdl_k, mdl_mn;
-    if (!make_map(&mdl_k, a.dL, vc_this, rows_cap, a.vc, TK, TM)) return DRK_ERR_CUDA;
-    if (!make_map(&mdl_mn, a.dL, vc_this, rows_cap, a.vc, 64, TK)) return DRK_ERR_CUDA;
+    const CUtensorMap& mdl_k = plan.mdl_k[chunk];
+    const CUtensorMap& mdl_mn = plan.mdl_mn[chunk];
     {  // dL chunk = c (softmax - onehot), recomputed from hidden W^T
       UmmaParams p{};
       p.m_tiles = (int)ceil_div(a.T, TMC);
@@ -752,7 +866,7 @@ int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {
       p.id_off = a.id_off; p.id_width = a.V;
       p.ids = a.ids; p.lse = a.lse; p.coeff = a.coeff; p.dL = a.dL; p.vc = a.vc; p.status = a.status;
       p.rowmap = a.rowmap; p.n_rows = a.n_rows;
-      int rc = launch_mode<DL>(ctas, mh_k, mw_k, p, st);
+      int rc = launch_mode<DL>(ctas, plan.mh_k, plan.mw_k, p, st);
       if (rc != DRK_OK) return rc;
     }
     {  // dW[v0 : v0 + vc_this, :] (+)= dL^T hidden
@@ -767,7 +881,7 @@ int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {
       p.beta = a.dw_accumulate; p.out_bf16 = a.dw_dtype == DRK_BF16; p.in_bf16 = p.out_bf16;
       p.status = a.status;
       p.rowmap = a.rowmap; p.n_rows = a.n_rows;
-      int rc = launch_mode<DW>(ctas, mdl_mn, mh_mn, p, st);
+      int rc = launch_mode<DW>(ctas, mdl_mn, plan.mh_mn, p, st);
       if (rc != DRK_OK) return rc;
       if (a.chunk_events != nullptr)
         DRK_CUDA_CHECK(cudaEventRecord(static_cast<cudaEvent_t>(a.chunk_events[chunk]), st));
@@ -785,11 +899,18 @@ int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {
       else { p.C = dh_acc; p.out_bf16 = 0; }
       p.status = a.status;
       p.rowmap = a.rowmap; p.n_rows = a.n_rows;
-      int rc = launch_mode<DH>(ctas, mdl_k, mw_mn, p, st);
+      int rc = launch_mode<DH>(ctas, mdl_k, plan.mw_mn, p, st);
       if (rc != DRK_OK) return rc;
     }
   }
   return DRK_OK;
+}
+
+int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {
+  UmmaBwdPlan plan;
+  int rc = plan_umma_bwd(a, &plan);
+  if (rc != DRK_OK) return rc;
+  return enqueue_umma_bwd(plan, st);
 }
 
 }  // namespace drk

@@ -1,0 +1,28 @@
+// Host-side plans of the tcgen05 path: everything a call needs that can fail on the host (driver entry point,
+// kernel attributes, tensor-map encoding) is done while the plan is built, before anything is enqueued.
+#pragma once
+#include "common.cuh"
+#include <cuda.h>
+#include <vector>
+
+namespace drk {
+
+struct UmmaFwdPlan {
+  UmmaFwdArgs a;
+  CUtensorMap mh, mw;   // hidden (or the gathered rows) and W, K-major boxes
+};
+int plan_umma_fwd(const UmmaFwdArgs& a, UmmaFwdPlan* plan);       // enqueues nothing
+int enqueue_umma_fwd(const UmmaFwdPlan& plan, cudaStream_t st);
+
+struct UmmaBwdPlan {
+  UmmaBwdArgs a;
+  CUtensorMap mh_k, mw_k, mh_mn, mw_mn;       // gathered hidden rows and W, as K-major and as MN-major operands
+  std::vector<CUtensorMap> mdl_k, mdl_mn;     // the dL buffer per vocabulary chunk (the last chunk is narrower)
+};
+int plan_umma_bwd(const UmmaBwdArgs& a, UmmaBwdPlan* plan);       // enqueues nothing
+int enqueue_umma_bwd(const UmmaBwdPlan& plan, cudaStream_t st);
+
+// Tensor maps encoded so far by this process (cache misses); steady-state calls add none.
+uint64_t umma_map_encodes();
+
+}  // namespace drk

@@ -24,9 +24,10 @@ TOL_ADV_REL = 1e-6
 # Rejection sampling (Sec. 5.1) compares a segment's MEAN log-ratio with thresholds only 1e-3 either side
 # of zero, so the decision is checked with a tolerance on that mean, not with the per-token one.  Both sides
 # read bit-identical inputs; the device's log-probs carry fp32 accumulation and ex2.approx rounding of
-# roughly 1e-5 per token, of either sign, and the mean over a segment's tokens is smaller still.  5e-5 is a
-# few times the largest deviation of ln(seg_w) from the oracle's mean seen on any case (each run reports it).
-TOL_MRS_MEAN = 5e-5
+# roughly 1e-5 per token, of either sign, and the mean over a segment's tokens is smaller still.  1e-5 is six
+# times the largest deviation of ln(seg_w) from the oracle's mean measured on any case (1.7e-6 on the reduced
+# 14B-shaped batch, 5.4e-7 at full size, ~2e-7 for fp32 inputs; each run reports its own figure).
+TOL_MRS_MEAN = 1e-5
 # Largest admissible share of segments whose decision is within rounding of a threshold.
 MAX_AMBIGUOUS_FRAC = 0.10
 

@@ -194,3 +194,28 @@ def test_extreme_aspect_ratios(T, H, V, S):
         dev = run_device(case, make_params(lo, hi, veto, engine=engine, dh_dtype=B.DRK_BF16))
         assert dev["status"] == 0
         Hh.check_against_oracle(case, dev, lo, hi, veto)
+
+
+@pytest.mark.parametrize("engine", [B.DRK_ENGINE_AUTO, B.DRK_ENGINE_UMMA_1CTA])
+def test_steady_state_calls_encode_no_tensor_maps(engine):
+    # tensor maps depend on addresses and geometry only: a second call on the same buffers finds all of them
+    d = torch.device("cuda:0")
+    case = Hh.build_plain_case("maps", T=300, H=128, V=1500, dtype=torch.bfloat16, S=3, seed=31)
+    p = make_params(*OPEN, v_chunk=512, engine=engine)
+    bufs = B.PgLossBuffers(case.T, case.H, case.V, case.S, B.DRK_BF16, p, d)
+    ins = [t.to(d) for t in (case.hidden, case.W, case.ids, case.rollout_logp, case.loss_mask, case.cu, case.seg_adv)]
+    B.pg_loss_fwd_bwd(*ins, p, bufs)
+    torch.cuda.synchronize()
+    first = (bufs.loss.clone(), bufs.dW.clone(), bufs.dH.clone())
+    n = B.drk_tensor_map_encodes()
+    assert n > 0
+    B.pg_loss_fwd_bwd(*ins, p, bufs)
+    torch.cuda.synchronize()
+    assert B.drk_tensor_map_encodes() == n
+    assert torch.equal(bufs.loss, first[0]) and torch.equal(bufs.dW, first[1]) and torch.equal(bufs.dH, first[2])
+    # other buffers of the same sizes get maps of their own
+    bufs2 = B.PgLossBuffers(case.T, case.H, case.V, case.S, B.DRK_BF16, p, d)
+    B.pg_loss_fwd_bwd(*ins, p, bufs2)
+    torch.cuda.synchronize()
+    assert B.drk_tensor_map_encodes() > n
+    assert torch.equal(bufs2.dW, first[1]) and torch.equal(bufs2.dH, first[2])
