@@ -62,6 +62,13 @@ typedef enum {
   DRK_ENGINE_UMMA_1CTA = 2 /* bf16 inputs: tcgen05 kernels with one CTA per 128x256 tile           */
 } drk_engine;
 
+typedef enum {
+  DRK_SCHEDULE_DYNAMIC = 0, /* blocks draw their next work unit from a device-side counter as they finish one:
+                               the units in flight are always consecutive, so the blocks that share an operand
+                               panel through L2 stay together however unevenly they progress                */
+  DRK_SCHEDULE_STATIC = 1   /* unit u belongs to block u mod (number of blocks), fixed at launch           */
+} drk_schedule;
+
 /* Bits of the device status word. */
 #define DRK_STATUS_BAD_ID 1u       /* some ids[t] outside [0,V): that row's target logit reads as 0 */
 #define DRK_STATUS_BAD_SEGMENTS 2u /* cu_seqlens not non-decreasing within [0,T]: segment skipped   */
@@ -171,6 +178,9 @@ typedef struct {
                             forward pass is skipped: a caller that judged its samples on log-probs from a
                             separate forward (samples split over micro-batches) pays for the logits three times,
                             not four.  entropy is left untouched.  forward_rows must be 0                 */
+  int32_t schedule;      /* drk_schedule of the tensor-core kernels' work units; default DRK_SCHEDULE_DYNAMIC.
+                            Results are bit-identical either way (every unit's output is independent of
+                            which block computes it)                                                     */
 } drk_pg_params;
 
 void drk_pg_params_default(drk_pg_params* p); /* host pointer */

@@ -33,6 +33,9 @@ DRK_ENGINE_AUTO = 0
 DRK_ENGINE_SIMT = 1
 DRK_ENGINE_UMMA_1CTA = 2
 
+DRK_SCHEDULE_DYNAMIC = 0
+DRK_SCHEDULE_STATIC = 1
+
 DRK_STATUS_BAD_ID = 1
 DRK_STATUS_BAD_SEGMENTS = 2
 DRK_STATUS_NONFINITE = 4
@@ -56,6 +59,7 @@ class drk_pg_params(ctypes.Structure):
         ("dw_chunk_events", ctypes.POINTER(ctypes.c_void_p)),
         ("n_dw_chunk_events", ctypes.c_int32),
         ("reuse_forward", ctypes.c_int32),
+        ("schedule", ctypes.c_int32),
     ]
 
 

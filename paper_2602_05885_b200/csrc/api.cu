@@ -103,12 +103,14 @@ struct FwdWs {
   float* part;
   float* tgt;
   int nsplit;
+  int32_t* sched;   // work counter of the forward kernel (tensor-core path)
 };
 FwdWs carve_fwd(Carver& c, int64_t T, int V, bool simt, int engine) {
   FwdWs w;
   w.nsplit = simt ? simt_nsplit(T, V) : umma_nsplit(T, V, umma_ctas(engine), false);
   w.part = static_cast<float*>(c.take(sizeof(float) * 4 * (size_t)w.nsplit * (size_t)T));
   w.tgt = static_cast<float*>(c.take(sizeof(float) * (size_t)T));
+  w.sched = simt ? nullptr : static_cast<int32_t*>(c.take(sizeof(int32_t)));
   return w;
 }
 
@@ -124,6 +126,7 @@ struct BwdWs {
   int32_t* n_rows;
   int32_t* rowmap;
   __nv_bfloat16* hidden_c;
+  int32_t* sched;   // work counters of the backward kernels, three per vocabulary chunk
 };
 BwdWs carve_bwd(Carver& c, int64_t T, int H, int V, int S, bool simt, const drk_pg_params& p) {
   BwdWs w;
@@ -133,9 +136,10 @@ BwdWs carve_bwd(Carver& c, int64_t T, int H, int V, int S, bool simt, const drk_
   const size_t rows_cap = (size_t)(ceil_div(T, 256) * 256);   // dL also holds the zero rows that pad the last tile
   w.dL = c.take((simt ? 4 : 2) * (simt ? (size_t)T : rows_cap) * (size_t)w.vc);
   w.dH_acc = (p.dh_dtype == DRK_BF16) ? static_cast<float*>(c.take(sizeof(float) * (size_t)T * (size_t)H)) : nullptr;
-  w.blk_cnt = w.blk_off = w.n_rows = w.rowmap = nullptr;
+  w.blk_cnt = w.blk_off = w.n_rows = w.rowmap = w.sched = nullptr;
   w.hidden_c = nullptr;
   if (!simt) {
+    w.sched = static_cast<int32_t*>(c.take(sizeof(int32_t) * 3 * (size_t)ceil_div(V, w.vc)));
     const size_t nblk = (size_t)compact_blocks(T), len = (size_t)compact_map_len(T);
     w.blk_cnt = static_cast<int32_t*>(c.take(sizeof(int32_t) * nblk));
     w.blk_off = static_cast<int32_t*>(c.take(sizeof(int32_t) * nblk));
@@ -156,6 +160,7 @@ bool params_ok(const drk_pg_params& p) {
   if (p.forward_rows != 0 && p.forward_rows != 1) return false;
   if (p.reuse_forward != 0 && p.reuse_forward != 1) return false;
   if (p.reuse_forward == 1 && p.forward_rows != 0) return false;
+  if (p.schedule != DRK_SCHEDULE_DYNAMIC && p.schedule != DRK_SCHEDULE_STATIC) return false;
   if (p.n_dw_chunk_events < 0 || (p.dw_chunk_events == nullptr && p.n_dw_chunk_events != 0)) return false;
   if (std::isnan(p.mrs_lo) || std::isnan(p.mrs_hi) || std::isnan(p.veto_ratio)) return false;
   if (p.norm == DRK_NORM_EXPLICIT && !std::isfinite(p.explicit_scale)) return false;
@@ -165,10 +170,11 @@ bool params_ok(const drk_pg_params& p) {
 UmmaFwdArgs umma_fwd_args(const void* hidden, const void* W, const int32_t* ids, int64_t T, int H, int V, int engine,
                           const FwdWs& w, float* logp, float* lse, float* entropy, uint32_t* status,
                           const __nv_bfloat16* hidden_c, const int32_t* rowmap, const int32_t* n_rows, int id_off,
-                          float* stats) {
+                          float* stats, bool dynamic = true) {
   UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, w.part, w.tgt, w.nsplit, status, umma_ctas(engine), entropy,
                 hidden_c, rowmap, n_rows};
   a.id_off = id_off; a.stats = stats;
+  a.sched = dynamic ? w.sched : nullptr;
   return a;
 }
 
@@ -251,13 +257,15 @@ int loss_fwd_bwd_impl(const void* hidden, const void* W, int32_t in_dtype, const
     if (fwd_here) {
       rc = plan_umma_fwd(umma_fwd_args(hidden, W, ids, T, H, V, p.engine, fw, logp, lse, entropy, status,
                                        fwd_rows ? bw.hidden_c : nullptr, fwd_rows ? bw.rowmap : nullptr,
-                                       fwd_rows ? bw.n_rows : nullptr, 0, nullptr), &fplan);
+                                       fwd_rows ? bw.n_rows : nullptr, 0, nullptr,
+                                       p.schedule == DRK_SCHEDULE_DYNAMIC), &fplan);
       if (rc != DRK_OK) return fail(rc);
     }
     UmmaBwdArgs b{hidden, W, ids, T, H, V, lse, bw.coeff, static_cast<__nv_bfloat16*>(bw.dL), bw.vc,
                   dH, p.dh_dtype, bw.dH_acc, dW, p.dw_dtype, p.dw_accumulate, status, umma_ctas(p.engine),
                   bw.hidden_c, bw.rowmap, bw.n_rows, p.dw_chunk_events};
     b.id_off = id_off;
+    b.sched = p.schedule == DRK_SCHEDULE_DYNAMIC ? bw.sched : nullptr;
     rc = plan_umma_bwd(b, &bplan);
     if (rc != DRK_OK) return fail(rc);
   }
@@ -354,6 +362,7 @@ void drk_pg_params_default(drk_pg_params* p) {
   p->dw_chunk_events = nullptr;
   p->n_dw_chunk_events = 0;
   p->reuse_forward = 0;
+  p->schedule = DRK_SCHEDULE_DYNAMIC;
 }
 
 int drk_pg_bwd_chunks(int64_t T, int32_t H, int32_t V, int32_t in_dtype, const drk_pg_params* pp, int32_t* v_chunk) {
@@ -525,6 +534,6 @@ const char* drk_status_string(int s) {
   }
 }
 
-int drk_version(void) { return 100; }
+int drk_version(void) { return 101; }
 
 }  // extern "C"

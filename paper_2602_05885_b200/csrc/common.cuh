@@ -99,6 +99,7 @@ struct UmmaFwdArgs {
   // optional: evaluate only the rows listed in rowmap (gathered into hidden_c); others are left untouched
   const __nv_bfloat16* hidden_c; const int32_t* rowmap; const int32_t* n_rows;
   int id_off = 0; float* stats = nullptr;   // vocabulary-range mode, as in SimtFwdArgs
+  int32_t* sched = nullptr;                 // one work counter (dynamic schedule) or null (static)
 };
 int umma_nsplit(int64_t T, int V, int ctas, bool frugal);
 int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st);
@@ -110,6 +111,7 @@ struct UmmaBwdArgs {
   const __nv_bfloat16* hidden_c; const int32_t* rowmap; const int32_t* n_rows;  // compacted rows
   void* const* chunk_events;  // optional cudaEvent_t per vocabulary chunk, recorded when its dW rows are final
   int id_off = 0;             // W holds columns [id_off, id_off + V) of a larger vocabulary
+  int32_t* sched = nullptr;   // three work counters per vocabulary chunk (dynamic schedule) or null (static)
 };
 int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st);
 

@@ -71,12 +71,13 @@ extern "C" int drk_pg_logprob_fwd_noalloc(const void* hidden, const void* W, int
   const bool simt = (in_dtype == DRK_F32) || (engine == DRK_ENGINE_SIMT);
   if (!simt && (H % 8) != 0) return DRK_ERR_UNSUPPORTED;
 
-  // scratch layout: partials [nsplit, T, 4] floats, then target logits [T] floats, each 256-aligned
+  // scratch layout: partials [nsplit, T, 4] floats, target logits [T] floats, one work counter; each 256-aligned
   const int ctas = engine == DRK_ENGINE_UMMA_1CTA ? 1 : 2;
   const int nsplit = simt ? simt_nsplit(T, V) : umma_nsplit(T, V, ctas, true);
   const size_t part_bytes = align_up(sizeof(float) * 4 * (size_t)nsplit * (size_t)T, 256);
   const size_t tgt_bytes = align_up(sizeof(float) * (size_t)T, 256);
-  if (part_bytes + tgt_bytes > kScratchBytes) return DRK_ERR_WORKSPACE;
+  const size_t sched_bytes = 256;   // the forward kernel's work counter (cleared by the launch code)
+  if (part_bytes + tgt_bytes + sched_bytes > kScratchBytes) return DRK_ERR_WORKSPACE;
 
   int dev = 0, major = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -93,6 +94,7 @@ extern "C" int drk_pg_logprob_fwd_noalloc(const void* hidden, const void* W, int
   UmmaFwdPlan plan;
   if (!simt) {   // kernel attributes and tensor maps (host only) before anything is enqueued
     UmmaFwdArgs a{hidden, W, ids, T, H, V, logp, lse, part, tgt, nsplit, status, ctas, nullptr, nullptr, nullptr, nullptr};
+    a.sched = reinterpret_cast<int32_t*>(static_cast<char*>(base) + part_bytes + tgt_bytes);
     rc = plan_umma_fwd(a, &plan);
     if (rc != DRK_OK) return rc;
   }

@@ -52,20 +52,36 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
+// The same test with acquire semantics at cluster scope: pairs with a remote arrive that releases data
+// written into this CTA's shared memory by the other CTA of the cluster.
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
 // Wait for the phase with the given parity to complete, for at most `limit_ns`.  Returns false if
 // the limit ran out or another thread of the block has already given up (*abort != 0); the first
 // thread to time out raises *abort so that every other waiter leaves within ~1k polls.  abort may
 // be null for a plain bounded wait.
+template <bool CLUSTER_ACQUIRE = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort,
                                           uint64_t limit_ns) {
+  auto test = [&]() { return CLUSTER_ACQUIRE ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
 #pragma unroll 1
   for (int i = 0; i < 64; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
+    if (test()) return true;
   const uint64_t t0 = globaltimer_ns();
   uint32_t polls = 0;
 #pragma unroll 1
   for (;;) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (test()) return true;
     if ((++polls & 0x3ffu) == 0) {
       if (abort != nullptr && *abort) return false;
       if (globaltimer_ns() - t0 > limit_ns) {
@@ -181,6 +197,15 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t bar, uint32_t cta) {
       "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
       "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
       ::"r"(bar), "r"(cta)
+      : "memory");
+}
+// Store a 32-bit word at the same shared-memory offset in CTA `cta` of the cluster.
+__device__ __forceinline__ void st_shared_remote(uint32_t addr, uint32_t cta, uint32_t value) {
+  asm volatile(
+      "{\n\t.reg .b32 ra;\n\t"
+      "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
+      "st.shared::cluster.u32 [ra], %2;\n\t}"
+      ::"r"(addr), "r"(cta), "r"(value)
       : "memory");
 }
 // Tile load issued by either CTA of a pair into its own shared memory; the transaction bytes are

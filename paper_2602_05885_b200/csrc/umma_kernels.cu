@@ -24,6 +24,7 @@
 #include <atomic>
 #include <math_constants.h>
 #include <mutex>
+#include <unordered_map>
 
 namespace drk {
 
@@ -45,8 +46,9 @@ constexpr int RING_BYTES = DRK_RING_KB * 1024;  // operand ring: 4 stages of 48 
 constexpr int MAX_STAGES = 8;
 constexpr int SUB_BYTES = 64 * TK * 2;    // one 64-wide MN-major box: 64 k-rows x 128 B
 constexpr int NUM_THREADS = 192;
-constexpr int NUM_BARS = 2 * MAX_STAGES + 5;
-constexpr int SMEM_BYTES = RING_BYTES + 1024 /*alignment slack*/ + NUM_BARS * 8 + 16;
+constexpr int SCHED_SLOTS = 4;            // work units announced ahead of their use (dynamic schedule)
+constexpr int NUM_BARS = 2 * MAX_STAGES + 5 + 2 * SCHED_SLOTS;
+constexpr int SMEM_BYTES = RING_BYTES + 1024 /*alignment slack*/ + NUM_BARS * 8 + 16 + 4 * SCHED_SLOTS;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;  // 2 s: far above any legitimate wait
 constexpr uint64_t DRAIN_LIMIT_NS = 20000000ull;   // 20 ms per outstanding copy when giving up
 constexpr float kLog2e = 1.4426950408889634f;
@@ -79,6 +81,10 @@ struct UmmaParams {
   // rowmap; their number is n_rows[0] (n_rows[1] = rounded up to 256), known on the device only.
   const int32_t* rowmap;
   const int32_t* n_rows;
+  // Dynamic schedule: a zeroed counter from which the blocks (CTA pairs) draw their next work unit as they
+  // finish one, so that the units in flight are always consecutive ones.  Null: unit u goes to block
+  // u mod (number of blocks).
+  int32_t* sched;
 };
 
 struct Unit {
@@ -110,12 +116,13 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 // Warp-collective bounded wait: all 32 lanes poll, and leave together.
+template <bool CLUSTER_ACQUIRE = false>
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort, int lane) {
   uint64_t t0 = 0;
   uint32_t polls = 0;
 #pragma unroll 1
   for (;;) {
-    const bool done = ptx::mbar_try_wait(bar, parity);
+    const bool done = CLUSTER_ACQUIRE ? ptx::mbar_try_wait_cluster(bar, parity) : ptx::mbar_try_wait(bar, parity);
     if (__all_sync(0xffffffffu, done)) return true;
     if ((++polls & 0x3ffu) == 0) {
       if (t0 == 0) t0 = ptx::globaltimer_ns();
@@ -211,8 +218,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + 2 + a); };
   const uint32_t done_bar = bar_base + 8u * (2 * MAX_STAGES + 4);
+  auto ufull_bar = [&](int s) { return bar_base + 8u * (2 * MAX_STAGES + 5 + s); };
+  auto uempty_bar = [&](int s) { return bar_base + 8u * (2 * MAX_STAGES + 5 + SCHED_SLOTS + s); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NUM_BARS);
   volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* unit_slot = reinterpret_cast<volatile int*>(tmem_slot + 4);   // [SCHED_SLOTS]
+  const uint32_t unit_slot_addr = ptx::smem_u32(tmem_slot + 4);
 
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
   const int lane = threadIdx.x & 31;
@@ -243,6 +254,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       ptx::mbar_init(tempty_bar(a), 4 * CTAS);
     }
     ptx::mbar_init(done_bar, 1);
+    for (int q = 0; q < SCHED_SLOTS; ++q) {
+      ptx::mbar_init(ufull_bar(q), 1);
+      // readers of a published unit: MMA thread and four epilogue warps in the even CTA; the producer
+      // thread and four epilogue warps in the odd one.  All of them release the slot in the even CTA.
+      ptx::mbar_init(uempty_bar(q), 5 * CTAS);
+    }
     *abort = 0;
     ptx::fence_barrier_init();
   }
@@ -260,6 +277,26 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // ---- work feed -------------------------------------------------------------------------------
+  // Static: the n-th unit of this block is first_unit + n * unit_stride.  Dynamic (p.sched): the even CTA's
+  // producer thread draws unit numbers from the global counter and announces the n-th one in slot
+  // n % SCHED_SLOTS of both CTAs' shared memory; every other role reads it there and releases the slot.
+  const bool dynamic = (p.sched != nullptr);
+  auto static_unit = [&](uint32_t n) {
+    const int64_t u = (int64_t)first_unit + (int64_t)n * unit_stride;
+    return u < num_units ? (int)u : -1;
+  };
+  // one thread: wait for the n-th announcement, read it, release the slot; -2 on a timed-out wait
+  auto take_unit = [&](uint32_t n) -> int {
+    if (!dynamic) return static_unit(n);
+    const int slot = n % SCHED_SLOTS;
+    if (!ptx::mbar_wait<true>(ufull_bar(slot), (n / SCHED_SLOTS) & 1u, abort, WAIT_LIMIT_NS)) return -2;
+    const int u = unit_slot[slot];
+    if (CTAS == 2 && !leader) ptx::mbar_arrive_remote(uempty_bar(slot), 0);
+    else ptx::mbar_arrive(uempty_bar(slot));
+    return u;
+  };
+
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -271,7 +308,38 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if constexpr (CTAS == 2) ptx::tma_load_2d_pair(dst, map, bar, x, y);
         else ptx::tma_load_2d(dst, map, bar, x, y);
       };
-      for (int u = first_unit; u < num_units && ok; u += unit_stride) {
+      // Even CTA, dynamic schedule: announce the n-th unit of this block to every other role of both CTAs.
+      auto announce = [&](uint32_t n, int u) -> bool {
+        const int slot = n % SCHED_SLOTS;
+        if (!ptx::mbar_wait(uempty_bar(slot), ((n / SCHED_SLOTS) & 1u) ^ 1u, abort, WAIT_LIMIT_NS)) return false;
+        unit_slot[slot] = u;
+        if constexpr (CTAS == 2) {
+          ptx::st_shared_remote(unit_slot_addr + 4u * slot, 1, (uint32_t)u);
+          ptx::mbar_arrive_remote(ufull_bar(slot), 1);   // release at cluster scope: orders the store above
+        }
+        ptx::mbar_arrive(ufull_bar(slot));
+        return true;
+      };
+      auto drawn = [&](int v) { return (int64_t)v + unit_stride < num_units ? v + unit_stride : -1; };
+      const bool feeder = dynamic && leader;
+      uint32_t seq = 0;
+      int u = -1, u_next = -1;
+      if (feeder) {
+        // the first unit is the block's own index; the counter hands out the units behind the first round.
+        // Units are announced one ahead, so that the other CTA's producer never waits for this one's loads.
+        u = static_unit(0);
+        if (u >= 0) u_next = drawn(atomicAdd(p.sched, 1));
+        ok = announce(0, u);
+      } else {
+        u = take_unit(0);
+      }
+      while (u >= 0 && ok) {
+        int pending = -1;
+        bool drew = false;
+        if (feeder) {
+          if (!announce(seq + 1, u_next)) { ok = false; break; }
+          if (u_next >= 0) { pending = atomicAdd(p.sched, 1); drew = true; }   // consumed after this unit's loads
+        }
         const Unit un = decode_unit(p, m_tiles, u);
         const int a_row = (un.m * CTAS + cta_rank) * TM;   // first A row (M index) of this CTA
         for (int n = un.n_begin; n < un.n_end && ok; ++n) {
@@ -304,7 +372,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             ++it;
           }
         }
+        ++seq;
+        if (feeder) { u = u_next; u_next = drew ? drawn(pending) : -1; }
+        else u = take_unit(seq);
       }
+      if (u == -2) ok = false;
       if (!ok && leader) {
         // wait (bounded) for the copies still in flight before the block leaves (a pair's loads are
         // all credited to the even CTA's barriers; the odd CTA waits for its peer at the cluster barrier)
@@ -321,7 +393,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       auto commit = [&](uint32_t bar) {
         if constexpr (CTAS == 2) ptx::mma_commit_pair(bar, (uint16_t)3); else ptx::mma_commit(bar);
       };
-      for (int u = first_unit; u < num_units && ok; u += unit_stride) {
+      uint32_t un_seq = 0;
+      int u = take_unit(0);
+      for (; u >= 0 && ok; u = take_unit(++un_seq)) {
         const Unit un = decode_unit(p, m_tiles, u);
         for (int n = un.n_begin; n < un.n_end && ok; ++n) {
           const int acc = tc & 1;
@@ -357,7 +431,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           commit(tfull_bar(acc));  // accumulator complete (in both CTAs)
           ++tc;
         }
+        if (!ok) break;
       }
+      if (u == -2) ok = false;
       if (!ok) {
         if constexpr (CTAS == 2) ptx::mma_commit_pair(done_bar, (uint16_t)1); else ptx::mma_commit(done_bar);
         ptx::mbar_wait(done_bar, 0, nullptr, DRAIN_LIMIT_NS);
@@ -368,7 +444,21 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int q = warp & 3;  // tensor-memory lane quarter this warp may read
     uint32_t tc = 0;
     bool ok = true;
-    for (int u = first_unit; u < num_units && ok; u += unit_stride) {
+    // warp-collective form of take_unit
+    auto take_unit_warp = [&](uint32_t n) -> int {
+      if (!dynamic) return static_unit(n);
+      const int slot = n % SCHED_SLOTS;
+      if (!mbar_wait_warp<true>(ufull_bar(slot), (n / SCHED_SLOTS) & 1u, abort, lane)) return -2;
+      const int u = unit_slot[slot];
+      __syncwarp();
+      if (lane == 0) {
+        if (CTAS == 2 && !leader) ptx::mbar_arrive_remote(uempty_bar(slot), 0);
+        else ptx::mbar_arrive(uempty_bar(slot));
+      }
+      return u;
+    };
+    uint32_t un_seq = 0;
+    for (int u = take_unit_warp(0); u >= 0 && ok; u = take_unit_warp(++un_seq)) {
       const Unit un = decode_unit(p, m_tiles, u);
       const int64_t row = ((int64_t)un.m * CTAS + cta_rank) * TM + q * 32 + lane;
       bool row_ok = row < rows;
@@ -559,7 +649,8 @@ EncodeTiledFn get_encode_fn() {
 
 // Tensor maps depend on the address and geometry only, never on the contents, so a map encoded once serves
 // every later call on the same buffer: a steady-state training step (same W, hidden and workspace pointers)
-// encodes nothing.  Small direct-mapped table with four probes, shared by all threads.
+// encodes nothing.  One table for the process, shared by all threads; emptied when it reaches kMapLimit
+// entries (a caller cycling through thousands of distinct buffers simply re-encodes).
 struct MapKey {
   const void* base; uint64_t inner, outer, pitch_bytes; uint32_t box_inner, box_outer, dtype;
   bool operator==(const MapKey& o) const {
@@ -567,19 +658,22 @@ struct MapKey {
            box_inner == o.box_inner && box_outer == o.box_outer && dtype == o.dtype;
   }
 };
-struct MapEntry { MapKey key; CUtensorMap map; bool used; };
-constexpr int kMapTable = 512;
+struct MapKeyHash {
+  size_t operator()(const MapKey& k) const {
+    uint64_t h = reinterpret_cast<uintptr_t>(k.base) * 0x9E3779B97F4A7C15ull;
+    h ^= (k.inner + 0x632BE59BD9B4E019ull) * 0xFF51AFD7ED558CCDull;
+    h ^= (k.outer + (h >> 29)) * 0xC4CEB9FE1A85EC53ull;
+    h ^= ((uint64_t)k.box_inner << 40) ^ ((uint64_t)k.box_outer << 20) ^ k.dtype ^ (k.pitch_bytes * 0x2545F4914F6CDD1Dull);
+    return (size_t)(h ^ (h >> 32));
+  }
+};
+constexpr size_t kMapLimit = 8192;
 std::mutex g_map_mu;
-MapEntry g_map_table[kMapTable] = {};
-std::atomic<uint64_t> g_map_encodes{0};
-
-size_t map_hash(const MapKey& k) {
-  uint64_t h = reinterpret_cast<uintptr_t>(k.base) * 0x9E3779B97F4A7C15ull;
-  h ^= (k.inner + 0x632BE59BD9B4E019ull) * 0xFF51AFD7ED558CCDull;
-  h ^= (k.outer + (h >> 29)) * 0xC4CEB9FE1A85EC53ull;
-  h ^= ((uint64_t)k.box_inner << 40) ^ ((uint64_t)k.box_outer << 20) ^ k.dtype ^ (k.pitch_bytes * 0x2545F4914F6CDD1Dull);
-  return (size_t)((h ^ (h >> 32)) % kMapTable);
+std::unordered_map<MapKey, CUtensorMap, MapKeyHash>& map_table() {
+  static auto* t = new std::unordered_map<MapKey, CUtensorMap, MapKeyHash>();   // never destroyed: no exit-order issues
+  return *t;
 }
+std::atomic<uint64_t> g_map_encodes{0};
 
 // Row-major matrix [outer, inner] of 2-byte (bf16) or 4-byte (fp32) elements with row pitch `pitch_elems`;
 // box = box_inner x box_outer, 128-byte swizzle, zero fill outside the extents on loads (stores are clipped).
@@ -589,13 +683,11 @@ bool make_map_typed(CUtensorMap* m, const void* base, uint64_t inner, uint64_t o
   if (!fn) return false;
   const uint32_t esz = f32 ? 4 : 2;
   const MapKey key{base, inner, outer, pitch_elems * esz, box_inner, box_outer, f32 ? 1u : 0u};
-  const size_t h = map_hash(key);
   {
     std::lock_guard<std::mutex> lock(g_map_mu);
-    for (int i = 0; i < 4; ++i) {
-      const MapEntry& e = g_map_table[(h + i) % kMapTable];
-      if (e.used && e.key == key) { *m = e.map; return true; }
-    }
+    auto& t = map_table();
+    auto it = t.find(key);
+    if (it != t.end()) { *m = it->second; return true; }
   }
   cuuint64_t dims[2] = {inner, outer};
   cuuint64_t strides[1] = {pitch_elems * esz};
@@ -607,12 +699,9 @@ bool make_map_typed(CUtensorMap* m, const void* base, uint64_t inner, uint64_t o
     return false;
   g_map_encodes.fetch_add(1, std::memory_order_relaxed);
   std::lock_guard<std::mutex> lock(g_map_mu);
-  int slot = (int)h;
-  for (int i = 0; i < 4; ++i)
-    if (!g_map_table[(h + i) % kMapTable].used) { slot = (int)((h + i) % kMapTable); break; }
-  g_map_table[slot].key = key;
-  g_map_table[slot].map = *m;
-  g_map_table[slot].used = true;
+  auto& t = map_table();
+  if (t.size() >= kMapLimit) t.clear();
+  t.emplace(key, *m);
   return true;
 }
 
@@ -802,6 +891,8 @@ int enqueue_umma_fwd(const UmmaFwdPlan& plan, cudaStream_t st) {
   p.ids = a.ids; p.part = a.part; p.tgt = a.tgt; p.status = a.status;
   p.want_entropy = a.entropy != nullptr || a.stats != nullptr;   // the statistics carry the same third sum
   p.rowmap = a.rowmap; p.n_rows = a.n_rows;
+  p.sched = a.sched;
+  if (a.sched != nullptr) DRK_CUDA_CHECK(cudaMemsetAsync(a.sched, 0, sizeof(int32_t), st));
   int rc = launch_mode<FWD>(ctas, plan.mh, plan.mw, p, st);
   if (rc != DRK_OK) return rc;
   if (a.stats != nullptr)
@@ -851,6 +942,8 @@ int enqueue_umma_bwd(const UmmaBwdPlan& plan, cudaStream_t st) {
   // rows that are not in the compacted set keep this zero
   DRK_CUDA_CHECK(cudaMemsetAsync(a.dH, 0, (size_t)a.T * a.H * (a.dh_dtype == DRK_BF16 ? 2 : 4), st));
   const int n_chunks = (int)ceil_div(a.V, a.vc);
+  // one work counter per launch (three per vocabulary chunk), all cleared by one memset
+  if (a.sched != nullptr) DRK_CUDA_CHECK(cudaMemsetAsync(a.sched, 0, sizeof(int32_t) * 3 * (size_t)n_chunks, st));
   int chunk = 0;
   for (int v0 = 0; v0 < a.V; v0 += a.vc, ++chunk) {
     const int vc_this = a.V - v0 < a.vc ? a.V - v0 : a.vc;
@@ -866,6 +959,7 @@ int enqueue_umma_bwd(const UmmaBwdPlan& plan, cudaStream_t st) {
       p.id_off = a.id_off; p.id_width = a.V;
       p.ids = a.ids; p.lse = a.lse; p.coeff = a.coeff; p.dL = a.dL; p.vc = a.vc; p.status = a.status;
       p.rowmap = a.rowmap; p.n_rows = a.n_rows;
+      p.sched = a.sched ? a.sched + 3 * chunk : nullptr;
       int rc = launch_mode<DL>(ctas, plan.mh_k, plan.mw_k, p, st);
       if (rc != DRK_OK) return rc;
     }
@@ -881,6 +975,7 @@ int enqueue_umma_bwd(const UmmaBwdPlan& plan, cudaStream_t st) {
       p.beta = a.dw_accumulate; p.out_bf16 = a.dw_dtype == DRK_BF16; p.in_bf16 = p.out_bf16;
       p.status = a.status;
       p.rowmap = a.rowmap; p.n_rows = a.n_rows;
+      p.sched = a.sched ? a.sched + 3 * chunk + 1 : nullptr;
       int rc = launch_mode<DW>(ctas, mdl_mn, plan.mh_mn, p, st);
       if (rc != DRK_OK) return rc;
       if (a.chunk_events != nullptr)
@@ -899,6 +994,7 @@ int enqueue_umma_bwd(const UmmaBwdPlan& plan, cudaStream_t st) {
       else { p.C = dh_acc; p.out_bf16 = 0; }
       p.status = a.status;
       p.rowmap = a.rowmap; p.n_rows = a.n_rows;
+      p.sched = a.sched ? a.sched + 3 * chunk + 2 : nullptr;
       int rc = launch_mode<DH>(ctas, mdl_k, plan.mw_mn, p, st);
       if (rc != DRK_OK) return rc;
     }

@@ -8,7 +8,7 @@ from paper_2602_05885_b200 import binding as B
 
 def make_params(lo=None, hi=None, veto=None, norm=0, explicit_scale=1.0, dw_dtype=B.DRK_F32, dh_dtype=B.DRK_F32,
                 dw_accumulate=0, engine=B.DRK_ENGINE_AUTO, v_chunk=0, keep_from_caller=0, forward_rows=0,
-                reuse_forward=0):
+                reuse_forward=0, schedule=B.DRK_SCHEDULE_DYNAMIC):
     p = B.drk_pg_params_default()
     if lo is not None:
         p.mrs_lo = lo
@@ -26,6 +26,7 @@ def make_params(lo=None, hi=None, veto=None, norm=0, explicit_scale=1.0, dw_dtyp
     p.keep_from_caller = keep_from_caller
     p.forward_rows = forward_rows
     p.reuse_forward = reuse_forward
+    p.schedule = schedule
     return p
 
 

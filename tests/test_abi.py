@@ -40,8 +40,8 @@ def test_defaults_are_the_papers_constants():
     assert abs(p.mrs_lo - 0.999) < 1e-7 and abs(p.mrs_hi - 1.001) < 1e-7     # Sec. 5.1 acceptance band
     assert abs(p.veto_ratio - 1e-4) < 1e-10                                     # Sec. 5.1 token veto
     assert p.norm == B.DRK_NORM_KEPT_TOKENS and p.engine == B.DRK_ENGINE_AUTO
-    assert ctypes.sizeof(B.drk_pg_params) == 64 and p.keep_from_caller == 0 and p.forward_rows == 0
-    assert p.reuse_forward == 0
+    assert ctypes.sizeof(B.drk_pg_params) == 72 and p.keep_from_caller == 0 and p.forward_rows == 0
+    assert p.reuse_forward == 0 and p.schedule == B.DRK_SCHEDULE_DYNAMIC
     assert not p.dw_chunk_events and p.n_dw_chunk_events == 0
 
 

@@ -211,6 +211,12 @@ def test_results_are_reproducible_bit_for_bit(engine):
     b = run_device(case, p)
     for k in ("logp", "lse", "entropy", "seg_w", "seg_keep", "loss", "counters", "dH", "dW"):
         assert torch.equal(a[k], b[k]), k
+    # which block computes which work unit does not matter either: a fixed assignment gives the same bits
+    c = run_device(case, make_params(lo, hi, PAPER[2], engine=engine, v_chunk=2048, dh_dtype=B.DRK_BF16,
+                                     schedule=B.DRK_SCHEDULE_STATIC))
+    assert c["status"] == 0
+    for k in ("logp", "lse", "entropy", "seg_w", "seg_keep", "loss", "counters", "dH", "dW"):
+        assert torch.equal(a[k], c[k]), k
 
 
 def test_caller_retention_combined_with_mrs():
