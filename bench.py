@@ -389,9 +389,9 @@ def main():
         return int((per_seg * keep.long()).sum().item())
 
     fused_ms = time_fused(p, min(args.steps, 5))
-    # merge + 3 MRS + 4 compaction kernels are not GEMM launches (the FFMA path has no compaction; the
-    # vocabulary-parallel form has one more merge)
-    n_gemm_launches = fused_launches[0] - (8 if code == B.DRK_BF16 else 4) - (1 if vocab else 0)
+    # merge + 3 MRS + 4 compaction kernels + the dH scatter are not GEMM launches (the FFMA path has neither
+    # compaction nor scatter; the vocabulary-parallel form has one more merge)
+    n_gemm_launches = fused_launches[0] - (9 if code == B.DRK_BF16 else 4) - (1 if vocab else 0)
     Tc = backward_rows() if code == B.DRK_BF16 else T
     Tf = int(bufs.counters[1].item()) if (p.forward_rows == 1 and code == B.DRK_BF16) else T   # rows the forward ran on
     flops = (2.0 * Tf + 6.0 * Tc) * H * V

@@ -135,7 +135,10 @@ BwdWs carve_bwd(Carver& c, int64_t T, int H, int V, int S, bool simt, const drk_
   w.seg_stats = static_cast<double*>(c.take(sizeof(double) * 4 * (size_t)S));
   const size_t rows_cap = (size_t)(ceil_div(T, 256) * 256);   // dL also holds the zero rows that pad the last tile
   w.dL = c.take((simt ? 4 : 2) * (simt ? (size_t)T : rows_cap) * (size_t)w.vc);
-  w.dH_acc = (p.dh_dtype == DRK_BF16) ? static_cast<float*>(c.take(sizeof(float) * (size_t)T * (size_t)H)) : nullptr;
+  // tensor-core path: fp32 accumulator of dH over the compacted rows (whatever dH's own type); FFMA path: an
+  // fp32 copy of dH only when dH itself is bf16
+  if (!simt) w.dH_acc = static_cast<float*>(c.take(sizeof(float) * rows_cap * (size_t)H));
+  else w.dH_acc = (p.dh_dtype == DRK_BF16) ? static_cast<float*>(c.take(sizeof(float) * (size_t)T * (size_t)H)) : nullptr;
   w.blk_cnt = w.blk_off = w.n_rows = w.rowmap = w.sched = nullptr;
   w.hidden_c = nullptr;
   if (!simt) {

@@ -106,7 +106,8 @@ int launch_umma_fwd(const UmmaFwdArgs& a, cudaStream_t st);
 struct UmmaBwdArgs {
   const void* hidden; const void* W; const int32_t* ids; int64_t T; int H; int V;
   const float* lse; const float* coeff; __nv_bfloat16* dL /*[T*vc]*/; int vc;
-  void* dH; int dh_dtype; float* dH_acc; void* dW; int dw_dtype; int dw_accumulate; uint32_t* status;
+  void* dH; int dh_dtype; float* dH_acc /*fp32 [ceil256(T), H]: accumulator over the compacted rows*/;
+  void* dW; int dw_dtype; int dw_accumulate; uint32_t* status;
   int ctas;
   const __nv_bfloat16* hidden_c; const int32_t* rowmap; const int32_t* n_rows;  // compacted rows
   void* const* chunk_events;  // optional cudaEvent_t per vocabulary chunk, recorded when its dW rows are final
@@ -124,6 +125,9 @@ struct CompactArgs {
 int64_t compact_map_len(int64_t T);
 int compact_blocks(int64_t T);
 int launch_compact(const CompactArgs& a, cudaStream_t st);
+// dst[rowmap[r], :] = src[r, :] for the n_rows[0] compacted rows; src fp32 [*, H], dst fp32 or bf16 [T, H]
+int launch_scatter_rows(const float* src, int H, const int32_t* rowmap, const int32_t* n_rows, void* dst, bool dst_bf16,
+                        cudaStream_t st);
 // need[t] = 1 for loss-masked tokens inside a segment, else 0 (the rows whose log-prob the loss can use)
 int launch_need_rows(const uint8_t* loss_mask, const int32_t* cu, int64_t T, int S, float* need, cudaStream_t st);
 

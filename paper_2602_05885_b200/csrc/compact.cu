@@ -74,6 +74,42 @@ __global__ void __launch_bounds__(256) gather_kernel(const __nv_bfloat16* __rest
   }
 }
 
+// dst[rowmap[r], :] = src[r, :] (fp32 -> fp32 or bf16), eight elements per thread and step.
+__global__ void __launch_bounds__(256) scatter_rows_kernel(const float* __restrict__ src, int H,
+                                                           const int32_t* __restrict__ rowmap,
+                                                           const int32_t* __restrict__ n_rows, void* __restrict__ dst,
+                                                           int dst_bf16) {
+  const int cnt = n_rows[0];
+  const int vec_per_row = H / 8;
+  for (int r = blockIdx.x; r < cnt; r += gridDim.x) {
+    const int t = rowmap[r];
+    if (t < 0) continue;
+    const float4* s = reinterpret_cast<const float4*>(src + (size_t)r * H);
+    for (int i = threadIdx.x; i < vec_per_row; i += blockDim.x) {
+      const float4 a = s[2 * i], b = s[2 * i + 1];
+      if (dst_bf16) {
+        __nv_bfloat162 p0 = __floats2bfloat162_rn(a.x, a.y), p1 = __floats2bfloat162_rn(a.z, a.w);
+        __nv_bfloat162 p2 = __floats2bfloat162_rn(b.x, b.y), p3 = __floats2bfloat162_rn(b.z, b.w);
+        uint4 o;
+        o.x = *reinterpret_cast<uint32_t*>(&p0); o.y = *reinterpret_cast<uint32_t*>(&p1);
+        o.z = *reinterpret_cast<uint32_t*>(&p2); o.w = *reinterpret_cast<uint32_t*>(&p3);
+        reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(dst) + (size_t)t * H)[i] = o;
+      } else {
+        float4* d = reinterpret_cast<float4*>(static_cast<float*>(dst) + (size_t)t * H);
+        d[2 * i] = a;
+        d[2 * i + 1] = b;
+      }
+    }
+  }
+}
+
+int launch_scatter_rows(const float* src, int H, const int32_t* rowmap, const int32_t* n_rows, void* dst, bool dst_bf16,
+                        cudaStream_t st) {
+  scatter_rows_kernel<<<sm_count() * 8, 256, 0, st>>>(src, H, rowmap, n_rows, dst, dst_bf16 ? 1 : 0);
+  DRK_LAUNCHED();
+  return DRK_OK;
+}
+
 __global__ void __launch_bounds__(256) need_rows_kernel(const uint8_t* __restrict__ mask, const int32_t* __restrict__ cu,
                                                         int64_t T, float* __restrict__ need) {
   const int g = blockIdx.x;

@@ -48,7 +48,12 @@ constexpr int SUB_BYTES = 64 * TK * 2;    // one 64-wide MN-major box: 64 k-rows
 constexpr int NUM_THREADS = 192;
 constexpr int SCHED_SLOTS = 4;            // work units announced ahead of their use (dynamic schedule)
 constexpr int NUM_BARS = 2 * MAX_STAGES + 5 + 2 * SCHED_SLOTS;
-constexpr int SMEM_BYTES = RING_BYTES + 1024 /*alignment slack*/ + NUM_BARS * 8 + 16 + 4 * SCHED_SLOTS;
+// Output staging for the TMA stores of the backward's epilogues: per epilogue warp two boxes of 32 rows x 128
+// bytes (128B-swizzled), so that a box can be filled while the TMA unit still reads the previous one.
+constexpr int OUT_BOX_BYTES = 32 * 128;
+constexpr int OUT_STAGE_BYTES = 4 * 2 * OUT_BOX_BYTES;
+constexpr int SMEM_BYTES = RING_BYTES + OUT_STAGE_BYTES + 1024 /*alignment slack*/ + NUM_BARS * 8 + 16 + 4 * SCHED_SLOTS;
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory per block");
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;  // 2 s: far above any legitimate wait
 constexpr uint64_t DRAIN_LIMIT_NS = 20000000ull;   // 20 ms per outstanding copy when giving up
 constexpr float kLog2e = 1.4426950408889634f;
@@ -76,6 +81,11 @@ struct UmmaParams {
   const void* C_in;
   int64_t ldc;
   int beta, out_bf16, in_bf16;
+  // How the epilogue of DL / DW / DH writes its tile: 0 = from registers (16-byte stores per thread, with a
+  // read-modify-write when beta is set); 1 = staged in shared memory and stored by the TMA unit through the
+  // output tensor map; 2 = the same with an element-wise add at the memory side (fp32 accumulation without
+  // the SM ever loading the old values).
+  int out_tma;
   uint32_t* status;
   // Compacted backward: the row dimension (M for DL and DH, K for DW) runs over the rows listed in
   // rowmap; their number is n_rows[0] (n_rows[1] = rounded up to 256), known on the device only.
@@ -109,6 +119,8 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+
+__device__ __forceinline__ uint32_t raw_bits(float v) { return __float_as_uint(v); }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -194,7 +206,7 @@ __device__ __forceinline__ void store_row_chunk(const UmmaParams& p, int64_t row
 template <int MODE, int CTAS>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                 const UmmaParams p) {
+                 const __grid_constant__ CUtensorMap tmC, const UmmaParams p) {
   constexpr bool A_MN = (MODE == DW);
   constexpr bool B_MN = (MODE == DW || MODE == DH);
   constexpr uint32_t IDESC = ptx::make_idesc_bf16(TM * CTAS, TN, A_MN ? 1 : 0, B_MN ? 1 : 0);
@@ -211,8 +223,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
   uint8_t* smem = smem_raw + pad;
   const uint32_t smem_base = raw_addr + pad;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + RING_BYTES);
-  const uint32_t bar_base = smem_base + RING_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + RING_BYTES + OUT_STAGE_BYTES);
+  const uint32_t bar_base = smem_base + RING_BYTES + OUT_STAGE_BYTES;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (MAX_STAGES + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + a); };
@@ -457,10 +469,40 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
       return u;
     };
+    // TMA-written outputs: this warp's two staging boxes, and how many boxes it has handed over so far
+    const uint32_t out_stage = smem_base + RING_BYTES + (uint32_t)(warp - 2) * 2 * OUT_BOX_BYTES;
+    const uint32_t out_row = out_stage + (uint32_t)lane * 128u;   // this lane's 128-byte row within box 0
+    uint32_t boxes = 0;
+    if constexpr (MODE != FWD) {
+      if (p.out_tma && lane == 0) ptx::prefetch_tensormap(&tmC);
+    }
+    // Box protocol (all lanes call, lane 0 talks to the TMA unit).  begin: the box to fill next was the source
+    // of the store issued two boxes ago, wait until that one has read it.  put: 16 bytes at chunk j of this
+    // lane's row, at the position the 128-byte swizzle gives it.  end: publish the writes to the async proxy
+    // and issue the store (or the add) of the box at tensor coordinates (x, y).
+    auto box_begin = [&]() {
+      if (lane == 0) ptx::bulk_wait_group_read<1>();
+      __syncwarp();
+    };
+    auto box_put = [&](int j, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+      ptx::st_shared_v4(out_row + (boxes & 1u) * OUT_BOX_BYTES + (uint32_t)((j ^ (lane & 7)) << 4), a, b, c, d);
+    };
+    auto box_end = [&](int x, int y) {
+      ptx::fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        const uint32_t src = out_stage + (boxes & 1u) * OUT_BOX_BYTES;
+        if (p.out_tma == 2) ptx::tma_reduce_add_2d(&tmC, src, x, y);
+        else ptx::tma_store_2d(&tmC, src, x, y);
+        ptx::bulk_commit_group();
+      }
+      ++boxes;
+    };
     uint32_t un_seq = 0;
     for (int u = take_unit_warp(0); u >= 0 && ok; u = take_unit_warp(++un_seq)) {
       const Unit un = decode_unit(p, m_tiles, u);
       const int64_t row = ((int64_t)un.m * CTAS + cta_rank) * TM + q * 32 + lane;
+      const int slab_row0 = (un.m * CTAS + cta_rank) * TM + q * 32;   // first row of this warp's 32-row slab
       bool row_ok = row < rows;
       // orow: the token this accumulator row belongs to (differs from row when rows are compacted)
       int64_t orow = row;
@@ -532,9 +574,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               run_m = m_new;
             }
           } else if constexpr (MODE == DL) {
-            if (row_ok && col < p.cols) {
+            // dL = c_t (softmax - onehot) for 32 columns of this lane's row
+            auto dl_values = [&]() {
               const int gcol = p.v0 + col;
-              if (c_t != 0.f) {
+              if (row_ok && c_t != 0.f) {
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                   const float pr = ex2(fmaf(x[j], kLog2e, -z2));
@@ -544,6 +587,22 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
                 for (int j = 0; j < 32; ++j) x[j] = 0.f;
               }
+            };
+            if (p.out_tma) {
+              // two 32-column blocks make one box of 64 bf16 columns (128 bytes per row); columns past the
+              // chunk's width are clipped by the store
+              const int pair_col = n * TN + (c & ~1) * 32;
+              if (slab_row0 < rows && pair_col < p.cols) {
+                dl_values();
+                if ((c & 1) == 0) box_begin();
+#pragma unroll
+                for (int qd = 0; qd < 4; ++qd)
+                  box_put((c & 1) * 4 + qd, pack_bf16(x[qd * 8 + 0], x[qd * 8 + 1]), pack_bf16(x[qd * 8 + 2], x[qd * 8 + 3]),
+                          pack_bf16(x[qd * 8 + 4], x[qd * 8 + 5]), pack_bf16(x[qd * 8 + 6], x[qd * 8 + 7]));
+                if (c & 1) box_end(pair_col, slab_row0);
+              }
+            } else if (row_ok && col < p.cols) {
+              dl_values();
               __nv_bfloat16* dst = p.dL + row * p.vc + col;
               if (col + 32 <= p.cols) {
                 uint4* d4 = reinterpret_cast<uint4*>(dst);
@@ -564,7 +623,28 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 for (int j = 0; j < 32; ++j) x[j] = 0.f;
               }
             }
-            if (row_ok && col < p.cols) store_row_chunk(p, orow, col, x);
+            if (p.out_tma) {
+              // rows past the output's extent (ragged vocabulary tail) and columns past H are clipped by the store
+              if (p.out_bf16) {
+                const int pair_col = n * TN + (c & ~1) * 32;
+                if (slab_row0 < rows && pair_col < p.cols) {
+                  if ((c & 1) == 0) box_begin();
+#pragma unroll
+                  for (int qd = 0; qd < 4; ++qd)
+                    box_put((c & 1) * 4 + qd, pack_bf16(x[qd * 8 + 0], x[qd * 8 + 1]), pack_bf16(x[qd * 8 + 2], x[qd * 8 + 3]),
+                            pack_bf16(x[qd * 8 + 4], x[qd * 8 + 5]), pack_bf16(x[qd * 8 + 6], x[qd * 8 + 7]));
+                  if (c & 1) box_end(pair_col, slab_row0);
+                }
+              } else if (slab_row0 < rows && col < p.cols) {
+                box_begin();
+#pragma unroll
+                for (int qd = 0; qd < 8; ++qd)
+                  box_put(qd, raw_bits(x[qd * 4 + 0]), raw_bits(x[qd * 4 + 1]), raw_bits(x[qd * 4 + 2]), raw_bits(x[qd * 4 + 3]));
+                box_end(col, slab_row0);
+              }
+            } else if (row_ok && col < p.cols) {
+              store_row_chunk(p, orow, col, x);
+            }
           }
         }
         // this warp has drained its quarter of the accumulator: tell the MMA issuer (even CTA)
@@ -583,6 +663,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           reinterpret_cast<float4*>(p.part)[(int64_t)un.j * p.T + row] = make_float4(run_m * kLn2, run_l, run_r, 0.f);
         }
       }
+    }
+    // every store this warp issued has been performed before the block (and its shared memory) goes away
+    if constexpr (MODE != FWD) {
+      if (lane == 0) ptx::bulk_wait_group<0>();
+      __syncwarp();
     }
   }
 
@@ -712,7 +797,7 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, 
 
 template <int MODE, int CTAS>
 __global__ void umma_gemm_kernel(const __grid_constant__ CUtensorMap, const __grid_constant__ CUtensorMap,
-                                 const UmmaParams);
+                                 const __grid_constant__ CUtensorMap, const UmmaParams);
 
 // How many two-CTA clusters of this kernel the device can hold at once (one CTA per SM); 0 if the query fails.
 int resident_pairs() {
@@ -771,8 +856,9 @@ int umma_prepare() {
   return state[dev] == 1 ? DRK_OK : DRK_ERR_CUDA;
 }
 
+// a, b: operand maps; c: the output map of the TMA-written epilogues (any valid map where out_tma is 0).
 template <int MODE, int CTAS>
-int launch_mode_ctas(const CUtensorMap& a, const CUtensorMap& b, UmmaParams p, cudaStream_t st) {
+int launch_mode_ctas(const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, UmmaParams p, cudaStream_t st) {
   p.num_units = p.m_tiles * p.nj;   // upper bound when the row count lives on the device
   if (p.num_units <= 0) return DRK_OK;
   auto kern = umma_gemm_kernel<MODE, CTAS>;
@@ -793,14 +879,15 @@ int launch_mode_ctas(const CUtensorMap& a, const CUtensorMap& b, UmmaParams p, c
   } else {
     cfg.gridDim = dim3(p.num_units < sm_count() ? p.num_units : sm_count());
   }
-  if (cudaLaunchKernelEx(&cfg, kern, a, b, p) != cudaSuccess) { (void)cudaGetLastError(); return DRK_ERR_CUDA; }
+  if (cudaLaunchKernelEx(&cfg, kern, a, b, c, p) != cudaSuccess) { (void)cudaGetLastError(); return DRK_ERR_CUDA; }
   DRK_LAUNCHED();
   return DRK_OK;
 }
 
 template <int MODE>
-int launch_mode(int ctas, const CUtensorMap& a, const CUtensorMap& b, const UmmaParams& p, cudaStream_t st) {
-  return ctas == 2 ? launch_mode_ctas<MODE, 2>(a, b, p, st) : launch_mode_ctas<MODE, 1>(a, b, p, st);
+int launch_mode(int ctas, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, const UmmaParams& p,
+                cudaStream_t st) {
+  return ctas == 2 ? launch_mode_ctas<MODE, 2>(a, b, c, p, st) : launch_mode_ctas<MODE, 1>(a, b, c, p, st);
 }
 
 }  // namespace
@@ -893,7 +980,7 @@ int enqueue_umma_fwd(const UmmaFwdPlan& plan, cudaStream_t st) {
   p.rowmap = a.rowmap; p.n_rows = a.n_rows;
   p.sched = a.sched;
   if (a.sched != nullptr) DRK_CUDA_CHECK(cudaMemsetAsync(a.sched, 0, sizeof(int32_t), st));
-  int rc = launch_mode<FWD>(ctas, plan.mh, plan.mw, p, st);
+  int rc = launch_mode<FWD>(ctas, plan.mh, plan.mw, plan.mh, p, st);
   if (rc != DRK_OK) return rc;
   if (a.stats != nullptr)
     return launch_shard_stats(a.part, a.tgt, a.ids, a.id_off, a.T, a.V, a.nsplit, a.stats, a.status, st);
@@ -925,12 +1012,22 @@ int plan_umma_bwd(const UmmaBwdArgs& a, UmmaBwdPlan* plan) {
   const int n_chunks = (int)ceil_div(a.V, a.vc);
   plan->mdl_k.resize(n_chunks);
   plan->mdl_mn.resize(n_chunks);
+  plan->mdl_out.resize(n_chunks);
+  plan->mdw_out.resize(n_chunks);
+  // Output boxes of the epilogues: 32 rows x 128 bytes (64 bf16 or 32 fp32 columns).
+  const bool dw_f32 = a.dw_dtype == DRK_F32;
+  plan->dw_out_tma = !a.dw_accumulate ? 1 : (dw_f32 ? 2 : 0);   // bf16 accumulation keeps the register path
   for (int c = 0; c < n_chunks; ++c) {
     const int v0 = c * a.vc;
     const int vc_this = a.V - v0 < a.vc ? a.V - v0 : a.vc;
     if (!make_map(&plan->mdl_k[c], a.dL, vc_this, rows_cap, a.vc, TK, TM)) return DRK_ERR_CUDA;
     if (!make_map(&plan->mdl_mn[c], a.dL, vc_this, rows_cap, a.vc, 64, TK)) return DRK_ERR_CUDA;
+    if (!make_map(&plan->mdl_out[c], a.dL, vc_this, rows_cap, a.vc, 64, 32)) return DRK_ERR_CUDA;
+    const void* dw_rows = (const char*)a.dW + (size_t)v0 * a.H * (dw_f32 ? 4 : 2);
+    if (!make_map_typed(&plan->mdw_out[c], dw_rows, a.H, vc_this, a.H, dw_f32 ? 32 : 64, 32, dw_f32)) return DRK_ERR_CUDA;
   }
+  // dH is accumulated in fp32 over the compacted rows and scattered to the tokens' rows at the end
+  if (!make_map_typed(&plan->mdh_out, a.dH_acc, a.H, rows_cap, a.H, 32, 32, true)) return DRK_ERR_CUDA;
   return DRK_OK;
 }
 
@@ -938,7 +1035,6 @@ int enqueue_umma_bwd(const UmmaBwdPlan& plan, cudaStream_t st) {
   const UmmaBwdArgs& a = plan.a;
   const int ctas = a.ctas == 2 ? 2 : 1;
   const int TMC = TM * ctas;   // rows of one work unit's tile
-  float* dh_acc = (a.dh_dtype == DRK_F32) ? (float*)a.dH : a.dH_acc;
   // rows that are not in the compacted set keep this zero
   DRK_CUDA_CHECK(cudaMemsetAsync(a.dH, 0, (size_t)a.T * a.H * (a.dh_dtype == DRK_BF16 ? 2 : 4), st));
   const int n_chunks = (int)ceil_div(a.V, a.vc);
@@ -959,8 +1055,9 @@ int enqueue_umma_bwd(const UmmaBwdPlan& plan, cudaStream_t st) {
       p.id_off = a.id_off; p.id_width = a.V;
       p.ids = a.ids; p.lse = a.lse; p.coeff = a.coeff; p.dL = a.dL; p.vc = a.vc; p.status = a.status;
       p.rowmap = a.rowmap; p.n_rows = a.n_rows;
+      p.out_tma = 1; p.out_bf16 = 1;
       p.sched = a.sched ? a.sched + 3 * chunk : nullptr;
-      int rc = launch_mode<DL>(ctas, plan.mh_k, plan.mw_k, p, st);
+      int rc = launch_mode<DL>(ctas, plan.mh_k, plan.mw_k, plan.mdl_out[chunk], p, st);
       if (rc != DRK_OK) return rc;
     }
     {  // dW[v0 : v0 + vc_this, :] (+)= dL^T hidden
@@ -973,33 +1070,32 @@ int enqueue_umma_bwd(const UmmaBwdPlan& plan, cudaStream_t st) {
       const size_t esz = a.dw_dtype == DRK_BF16 ? 2 : 4;
       p.C = (char*)a.dW + (size_t)v0 * a.H * esz; p.C_in = p.C; p.ldc = a.H;
       p.beta = a.dw_accumulate; p.out_bf16 = a.dw_dtype == DRK_BF16; p.in_bf16 = p.out_bf16;
+      p.out_tma = plan.dw_out_tma;
       p.status = a.status;
       p.rowmap = a.rowmap; p.n_rows = a.n_rows;
       p.sched = a.sched ? a.sched + 3 * chunk + 1 : nullptr;
-      int rc = launch_mode<DW>(ctas, mdl_mn, plan.mh_mn, p, st);
+      int rc = launch_mode<DW>(ctas, mdl_mn, plan.mh_mn, plan.mdw_out[chunk], p, st);
       if (rc != DRK_OK) return rc;
       if (a.chunk_events != nullptr)
         DRK_CUDA_CHECK(cudaEventRecord(static_cast<cudaEvent_t>(a.chunk_events[chunk]), st));
     }
-    {  // dH (+)= dL W[v0 : v0 + vc_this, :]
+    {  // dH_acc (+)= dL W[v0 : v0 + vc_this, :], over the compacted rows: stored by the first chunk, added to by the rest
       UmmaParams p{};
       p.m_tiles = (int)ceil_div(a.T, TMC);
       p.n_tiles = (int)ceil_div(a.H, TN);
       p.k_blocks = (int)ceil_div(vc_this, TK);
       p.nj = p.n_tiles; p.tiles_per_unit = 1; p.group_m = 32 / ctas;
       p.rows = a.T; p.cols = a.H; p.v0 = v0; p.T = a.T;
-      const bool last = (chunk == n_chunks - 1);
-      p.C_in = dh_acc; p.in_bf16 = 0; p.ldc = a.H; p.beta = chunk > 0;
-      if (last && a.dh_dtype == DRK_BF16) { p.C = a.dH; p.out_bf16 = 1; }
-      else { p.C = dh_acc; p.out_bf16 = 0; }
+      p.ldc = a.H; p.out_bf16 = 0; p.out_tma = chunk > 0 ? 2 : 1;
       p.status = a.status;
-      p.rowmap = a.rowmap; p.n_rows = a.n_rows;
+      p.rowmap = nullptr; p.n_rows = a.n_rows;
       p.sched = a.sched ? a.sched + 3 * chunk + 2 : nullptr;
-      int rc = launch_mode<DH>(ctas, mdl_k, plan.mw_mn, p, st);
+      int rc = launch_mode<DH>(ctas, mdl_k, plan.mw_mn, plan.mdh_out, p, st);
       if (rc != DRK_OK) return rc;
     }
   }
-  return DRK_OK;
+  // dH[rowmap[r], :] = dH_acc[r, :] in the requested type
+  return launch_scatter_rows(a.dH_acc, a.H, a.rowmap, a.n_rows, a.dH, a.dh_dtype == DRK_BF16, st);
 }
 
 int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {

@@ -18,6 +18,11 @@ struct UmmaBwdPlan {
   UmmaBwdArgs a;
   CUtensorMap mh_k, mw_k, mh_mn, mw_mn;       // gathered hidden rows and W, as K-major and as MN-major operands
   std::vector<CUtensorMap> mdl_k, mdl_mn;     // the dL buffer per vocabulary chunk (the last chunk is narrower)
+  // outputs written by the TMA unit in boxes of 32 rows x 128 bytes: the dL chunk, the chunk's rows of dW, and
+  // the fp32 accumulator of dH over the compacted rows
+  std::vector<CUtensorMap> mdl_out, mdw_out;
+  CUtensorMap mdh_out;
+  int dw_out_tma;                             // 1 store, 2 add (fp32 accumulation), 0 register path
 };
 int plan_umma_bwd(const UmmaBwdArgs& a, UmmaBwdPlan* plan);       // enqueues nothing
 int enqueue_umma_bwd(const UmmaBwdPlan& plan, cudaStream_t st);
