@@ -42,6 +42,47 @@ def measured_peaks():
     return dict(tflops=1400.0, burst=1590.0, hbm=6650.0, source="fallback")
 
 
+KERNEL_SOURCES = ["umma_kernels.cu", "umma.cuh", "umma_plan.cuh", "compact.cu", "api.cu", "common.cuh"]
+TRAFFIC_PROFILE = os.path.join(ROOT, "profiles", "umma_gemm_kernel_dram_traffic_model.md")
+
+
+def kernel_source_hash() -> str:
+    """sha256 over the sources that decide the tensor-core kernels' memory traffic (kernels, launch geometry)."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2602_05885_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def traffic_model(config: dict, rows_fwd: int, rows_bwd: int, n_chunks: int):
+    """DRAM bytes (read + write) of one fused call, from the tracked ncu summary.
+
+    The summary holds, per kernel instantiation, bytes = A + B * rows fitted to one-pass captures of
+    dram__bytes_read.sum + dram__bytes_write.sum at two reduced row counts (same H, V and chunk width as the
+    benchmark), together with the hash of the kernel sources and the configuration they were taken with.
+    Returns (bytes, note); bytes is None when the sources or the configuration differ from the capture's."""
+    import re
+    if not os.path.exists(TRAFFIC_PROFILE):
+        return None, "no tracked capture"
+    text = open(TRAFFIC_PROFILE).read()
+    m = re.search(r"```json\s*(\{.*?\})\s*```", text, flags=re.S)
+    if not m:
+        return None, "no model in the tracked capture"
+    model = json.loads(m.group(1))
+    if model.get("kernel_source_sha256") != kernel_source_hash():
+        return None, "kernel sources changed since the capture"
+    if any(model["config"].get(k) != v for k, v in config.items()) or model["config"].get("chunks") != n_chunks:
+        return None, "configuration differs from the capture's"
+    total = 0.0
+    for mode, rows in (("FWD", rows_fwd), ("DL", rows_bwd), ("DW", rows_bwd), ("DH", rows_bwd)):
+        total += model["bytes"][mode]["A"] + model["bytes"][mode]["B_per_row"] * rows
+    return total, (f"A + B*rows per kernel, fitted to one-pass ncu captures at {model['fit_rows']} rows "
+                   f"(checked at {model['check_rows']}: {model['check_error_pct']} % off), "
+                   f"profiles/{os.path.basename(TRAFFIC_PROFILE)}")
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -109,12 +150,12 @@ def run_reference(args):
     mask = wl.loss_mask.numpy()
     cu = wl.cu.numpy()
     adv = np.ones(wl.S)
-    lo, hi = wl.wide_band()
 
     def step():
+        # the benchmark's default: acceptance band open, veto off (every sample retained)
         G = O.returns(wl.reward.numpy(), wl.valid.numpy(), 1.0)
         O.trloo_advantage(G, wl.valid.numpy(), wl.prompt_of_rollout.numpy())
-        return O.pg_loss_fwd_bwd(hidden, W, ids, rl, mask, cu, adv, lo=lo, hi=hi)
+        return O.pg_loss_fwd_bwd(hidden, W, ids, rl, mask, cu, adv, lo=0.0, hi=float("inf"), veto=0.0)
 
     for _ in range(args.warmup):
         step()
@@ -147,12 +188,11 @@ def cpu_baseline(n_tok: int):
     wl = workload.build("qwen3-14b", "cpu", seed=2000, T_override=n_tok)
     hidden = wl.hidden.double().numpy()
     W = wl.W.double().numpy()
-    lo, hi = wl.wide_band()
     t0 = time.perf_counter()
     G = O.returns(wl.reward.numpy(), wl.valid.numpy(), 1.0)
     O.trloo_advantage(G, wl.valid.numpy(), wl.prompt_of_rollout.numpy())
     O.pg_loss_fwd_bwd(hidden, W, wl.ids.numpy(), wl.rollout_logp.double().numpy(), wl.loss_mask.numpy(),
-                      wl.cu.numpy(), np.ones(wl.S), lo=lo, hi=hi)
+                      wl.cu.numpy(), np.ones(wl.S), lo=0.0, hi=float("inf"), veto=0.0)
     dt = time.perf_counter() - t0
     return {"value": n_tok / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"one pass over {n_tok} packed tokens at full H=5120, V=151936 in {dt:.1f} s "
@@ -228,7 +268,11 @@ def main():
                          "(overlapped on a second stream); off by default: the loss path itself needs no collective")
     ap.add_argument("--engine", default="auto", choices=["auto", "1cta"],
                     help="auto: tcgen05 kernels on CTA pairs; 1cta: one CTA per tile")
-    ap.add_argument("--mrs", default="wide", choices=["wide", "paper", "off"])
+    ap.add_argument("--mrs", default="off", choices=["off", "wide", "paper"],
+                    help="off (default): the acceptance band is open and the veto disabled, so every loss-masked token "
+                         "goes through the backward (the full 8 T H V of work; the rejection kernels still run); "
+                         "wide: a band that retains about half of the samples; paper: [0.999, 1.001] and the 1e-4 veto, "
+                         "under which this workload's noise level rejects nearly every sample")
     ap.add_argument("--parallelism", default="data", choices=["data", "vocab"],
                     help="data: one micro-batch per rank, no collective on the loss path (weak scaling); "
                          "vocab: W split by rows over the ranks, one micro-batch for all (strong scaling)")
@@ -397,22 +441,26 @@ def main():
     flops = (2.0 * Tf + 6.0 * Tc) * H * V
     peaks = measured_peaks()
     achieved = flops / (fused_ms * 1e-3) / 1e12
-    # DRAM bytes (read + write) of one fused call, from a one-pass ncu capture of exactly this configuration
-    # with the kernels as they are; unknown (null) for any other configuration.
-    traffic = None
-    if (args.workload, T, args.mrs, args.dw_dtype, args.dh_dtype, args.v_chunk, args.engine, args.forward_rows,
-            args.parallelism) == ("qwen3-14b", 32768, "wide", "f32", "bf16", 0, "auto", "all", "data"):
-        traffic = 181.81e9
-    # the same call with rejection switched off: every loss-masked token goes through the backward
-    p_off = B.drk_pg_params_default()
-    ctypes_copy = [f[0] for f in p._fields_]
-    for f in ctypes_copy:
-        setattr(p_off, f, getattr(p, f))
-    p_off.mrs_lo, p_off.mrs_hi, p_off.veto_ratio = 0.0, float("inf"), 0.0
-    off_ms = time_fused(p_off, min(args.steps, 5))
-    Tc_off = backward_rows() if code == B.DRK_BF16 else T
-    off_tflops = (2.0 * Tf + 6.0 * Tc_off) * H * V / (off_ms * 1e-3) / 1e12
-    time_fused(p, 1)   # leave the outputs of the configured run in the buffers
+    n_chunks, vc_used = B.drk_pg_bwd_chunks(T, H, V, code, p)
+    traffic, traffic_note = traffic_model(dict(H=H, V=V_total, v_chunk=vc_used, dW=args.dw_dtype, dH=args.dh_dtype,
+                                               engine=args.engine, parallelism=args.parallelism, dtype="bf16" if
+                                               code == B.DRK_BF16 else "f32"), Tf, Tc, n_chunks)
+    # the same call with a band that retains about half of the samples: rows of rejected samples skip the backward
+    wide = None
+    if args.mrs == "off":
+        p_w = B.drk_pg_params_default()
+        for f, _ in p._fields_:
+            setattr(p_w, f, getattr(p, f))
+        p_w.mrs_lo, p_w.mrs_hi = wl.wide_band()
+        p_w.veto_ratio = B.drk_pg_params_default().veto_ratio
+        w_ms = time_fused(p_w, min(args.steps, 5))
+        Tc_w = backward_rows() if code == B.DRK_BF16 else T
+        w_tflops = (2.0 * Tf + 6.0 * Tc_w) * H * V / (w_ms * 1e-3) / 1e12
+        wide = {"call_ms": w_ms, "rows_in_backward": Tc_w, "tflops": w_tflops, "frac": w_tflops / peaks["tflops"],
+                "tokens_per_s": T / (w_ms * 1e-3),
+                "what": "same call, acceptance band exp(-+q) around 1 with q between the middle order statistics of the "
+                        "samples' |mean log-ratio| (about half retained), veto 1e-4"}
+        time_fused(p, 1)   # leave the outputs of the configured run in the buffers
 
     # ---------------------------------------------------------------- end to end with host buffers
     e2e = None
@@ -497,7 +545,9 @@ def main():
             "scaling": "strong" if vocab else "weak",
             "vs_baseline": None, "dtype": "bf16" if code == B.DRK_BF16 else "f32", "data": "synthetic",
             "config": {"workload": f"{wl.name}-shaped packed micro-batch", "T": T, "H": H, "V": V_total, "V_local": V, "segments": S,
-                       "rollout_batch": f"{R} rollouts x {Tmax} turns", "mrs": args.mrs,
+                       "rollout_batch": f"{R} rollouts x {Tmax} turns",
+                       "mrs": {"off": "band open, veto off: every loss-masked token goes through the backward (8 T H V)",
+                               "wide": "band retaining about half of the samples", "paper": "[0.999, 1.001], veto 1e-4"}[args.mrs],
                        "dW": args.dw_dtype, "dH": args.dh_dtype, "v_chunk": args.v_chunk or "default",
                        "engine": args.engine, "forward_rows": args.forward_rows,
                        "l2": "inputs exceed L2 (W alone is %.2f GB); no flush" % (V * H * 2 / 1e9),
@@ -507,18 +557,20 @@ def main():
                                        ("dW all-reduced per vocabulary chunk, overlapped" if args.sync_dw
                                         else "no collective on the loss path"))},
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s",
-                         "frac": achieved / peaks["tflops"], "traffic": traffic,
+                         "frac": achieved / peaks["tflops"], "traffic": traffic, "traffic_source": traffic_note,
                          "kernel": "umma_gemm_kernel (all four instantiations inside one drk_pg_loss_fwd_bwd call)",
                          "flops_per_call": flops, "call_ms": fused_ms, "gemm_launches_per_call": n_gemm_launches,
                          "flops_rule": "(2 T + 6 Tc) H V: forward over all T rows, backward over the Tc rows with "
                                        "a non-zero coefficient (rows of rejected or masked tokens are skipped)",
                          "rows_in_backward": Tc, "rows_in_forward": Tf,
-                         "no_rejection": {"call_ms": off_ms, "rows_in_backward": Tc_off, "tflops": off_tflops,
-                                          "frac": off_tflops / peaks["tflops"],
-                                          "tokens_per_s": T / (off_ms * 1e-3)},
                          "peak_source": f"bf16_tflops_sustained of {peaks['source']}",
-                         "frac_of_burst": achieved / peaks["burst"], "frac_of_nominal_2250": achieved / 2250.0},
-            "value_no_rejection": T / (off_ms * 1e-3),   # the fused call alone with every sample retained (all rows in the backward)
+                         "frac_of_burst": achieved / peaks["burst"], "frac_of_nominal_2250": achieved / 2250.0,
+                         # the chip's dense bf16 rate at the clock it actually ran at (nominal 2250 TFLOP/s at the
+                         # maximum SM clock, scaled by the median clock sampled during the timed region)
+                         "frac_of_nominal_at_sampled_clock": (achieved / (2250.0 * clocks["sm_mhz"] / clocks["sm_max_mhz"])
+                                                              if clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz")
+                                                              else None)},
+            "with_rejection_wide_band": wide,
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": n_launch, "clocks": clocks,
             "status_word": status, "counters": {"kept_tokens": counters[0], "masked_tokens": counters[1],
                                                 "kept_segments": counters[2], "vetoed_segments": counters[3]},
