@@ -328,6 +328,11 @@ def main():
         p.mrs_lo, p.mrs_hi, p.veto_ratio = 0.0, float("inf"), 0.0
     p.dw_dtype = B.DRK_BF16 if args.dw_dtype == "bf16" else B.DRK_F32
     p.dh_dtype = B.DRK_BF16 if args.dh_dtype == "bf16" else B.DRK_F32
+    # vocabulary parallel on several ranks: every rank's dH is a partial sum, and the parts cross the ranks in
+    # fp32; the requested bf16 is produced after the reduction
+    dh_bf16_after = vocab and world > 1 and p.dh_dtype == B.DRK_BF16
+    if dh_bf16_after:
+        p.dh_dtype = B.DRK_F32
     p.v_chunk = args.v_chunk
     p.engine = B.DRK_ENGINE_UMMA_1CTA if args.engine == "1cta" else B.DRK_ENGINE_AUTO
     p.forward_rows = 1 if args.forward_rows == "usable" else 0
@@ -340,6 +345,7 @@ def main():
     seg_turn = wl.seg_turn.to(torch.int32).contiguous()
     seg_adv = torch.empty(S, dtype=torch.float32, device=dev)
     stats = torch.empty((T, 4), dtype=torch.float32, device=dev)
+    dh_out = torch.empty((T, H), dtype=torch.bfloat16, device=dev) if dh_bf16_after else None
     stream = torch.cuda.current_stream()
     launches = [0]
     comm = None
@@ -357,13 +363,13 @@ def main():
     def step(hidden, ids, rl, mask, cu, out=None):
         o = out if out is not None else bufs
         B.drk_trloo_advantage(wl.reward, wl.valid, wl.prompt_of_rollout, R, Tmax, 1.0, B.DRK_BASELINE_TRLOO,
-                              ret, adv, gsize, stream)
+                              ret, adv, gsize, o.status, stream)
         launches[0] += B.drk_last_launch_count()
         B.drk_segment_advantages(adv, seg_rollout, seg_turn, R, Tmax, S, seg_adv, o.status, stream)
         launches[0] += B.drk_last_launch_count()
         if vocab:
             launches[0] += dp.vocab_parallel_loss_fwd_bwd(hidden, W_local, ids, rl, mask, cu, seg_adv, v_begin, V_total,
-                                                          p, o, stats, stream)
+                                                          p, o, stats, stream, dh_out)
             return
         B.drk_pg_loss_fwd_bwd(hidden, W_local, code, ids, rl, mask, cu, seg_adv, T, H, V, S, p, o.loss, o.logp,
                               o.lse, o.entropy, o.seg_w, o.seg_keep, o.counters, o.dH, o.dW,
@@ -412,7 +418,7 @@ def main():
             if vocab:      # this rank's two calls with the exchange between them
                 fused_launches[0] = dp.vocab_parallel_loss_fwd_bwd(wl.hidden, W_local, wl.ids, wl.rollout_logp,
                                                                    wl.loss_mask, wl.cu, seg_adv, v_begin, V_total, pp,
-                                                                   bufs, stats, stream)
+                                                                   bufs, stats, stream, dh_out)
             else:
                 B.drk_pg_loss_fwd_bwd(wl.hidden, W_local, code, wl.ids, wl.rollout_logp, wl.loss_mask, wl.cu, seg_adv,
                                       T, H, V, S, pp, bufs.loss, bufs.logp, bufs.lse, bufs.entropy, bufs.seg_w,

@@ -74,6 +74,10 @@ typedef enum {
 #define DRK_STATUS_BAD_SEGMENTS 2u /* cu_seqlens not non-decreasing within [0,T]: segment skipped   */
 #define DRK_STATUS_NONFINITE 4u    /* a non-finite log-sum-exp was produced                         */
 #define DRK_STATUS_TIMEOUT 8u      /* a bounded on-chip wait expired; results are invalid           */
+#define DRK_STATUS_BOUNDS 32u      /* checked build only (library compiled with -DDRK_BOUNDS_CHECK): an index
+                                      derived on the device fell outside its array; the access was skipped    */
+#define DRK_STATUS_BAD_GROUPS 16u  /* prompt_of_rollout decreases somewhere: a prompt's rollouts are not
+                                      contiguous, so its turn groups were split (Sec. 4.2 groups by prompt) */
 
 /*
  * Reward-to-go returns and turn-level advantages for a whole rollout batch
@@ -87,15 +91,19 @@ typedef enum {
  *
  * reward, valid, ret, adv, gsize are [R*Tmax] device arrays indexed i*Tmax+t;
  * prompt_of_rollout is [R] device, non-decreasing (rollouts of a prompt are
- * contiguous).  Invalid (i,t) get ret = adv = 0 and gsize = 0; valid ones get
- * gsize = group size.  Arithmetic is fp64 inside, outputs are rounded to fp32.
- * An all-equal group yields exactly 0.  R, Tmax >= 0 (0 enqueues nothing);
- * Tmax <= 64, else DRK_ERR_UNSUPPORTED.  gamma must lie in [0,1].
+ * contiguous): groups are the runs of equal values.  Where the array decreases,
+ * a prompt whose rollouts are scattered would silently fall into several groups,
+ * so that condition sets DRK_STATUS_BAD_GROUPS in *status (device uint32, OR-ed
+ * into; may be NULL to skip the check).  Invalid (i,t) get ret = adv = 0 and
+ * gsize = 0; valid ones get gsize = group size.  Arithmetic is fp64 inside,
+ * outputs are rounded to fp32.  An all-equal group yields exactly 0.
+ * R, Tmax >= 0 (0 enqueues nothing); Tmax <= 64, else DRK_ERR_UNSUPPORTED.
+ * gamma must lie in [0,1].
  */
 int drk_trloo_advantage(const float* reward, const uint8_t* valid,
                         const int32_t* prompt_of_rollout, int32_t R, int32_t Tmax,
                         float gamma, int32_t baseline, float* ret, float* adv,
-                        int32_t* gsize, void* stream);
+                        int32_t* gsize, uint32_t* status, void* stream);
 
 /*
  * Per-sample advantages of a packed micro-batch.  Every turn of a trajectory is one training sample
@@ -367,6 +375,8 @@ uint64_t drk_tensor_map_encodes(void);
 
 const char* drk_status_string(int status);
 int drk_version(void);
+/* 1 if this library was compiled with -DDRK_BOUNDS_CHECK (see DRK_STATUS_BOUNDS), else 0. */
+int drk_bounds_checked(void);
 
 #ifdef __cplusplus
 }

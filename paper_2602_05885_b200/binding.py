@@ -40,6 +40,8 @@ DRK_STATUS_BAD_ID = 1
 DRK_STATUS_BAD_SEGMENTS = 2
 DRK_STATUS_NONFINITE = 4
 DRK_STATUS_TIMEOUT = 8
+DRK_STATUS_BAD_GROUPS = 16
+DRK_STATUS_BOUNDS = 32
 
 
 class drk_pg_params(ctypes.Structure):
@@ -88,7 +90,9 @@ _lib: Optional[ctypes.CDLL] = None
 
 
 def library_path() -> str:
-    return _build.LIB_PATH
+    """The in-tree libdrk.so, or the build named by the environment variable DRK_LIBRARY (for instance the
+    checked build libdrk_check.so, whose kernels range-check every index they derive on the device)."""
+    return os.environ.get("DRK_LIBRARY") or _build.LIB_PATH
 
 
 def load() -> ctypes.CDLL:
@@ -109,7 +113,7 @@ def load() -> ctypes.CDLL:
     lib.drk_pg_bwd_chunks.restype = ctypes.c_int
     lib.drk_pg_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, ctypes.POINTER(drk_pg_params), i32]
     lib.drk_pg_workspace_bytes.restype = sz
-    lib.drk_trloo_advantage.argtypes = [vp, vp, vp, i32, i32, f32, i32, vp, vp, vp, vp]
+    lib.drk_trloo_advantage.argtypes = [vp, vp, vp, i32, i32, f32, i32, vp, vp, vp, vp, vp]
     lib.drk_trloo_advantage.restype = ctypes.c_int
     lib.drk_pg_logprob_fwd.argtypes = [vp, vp, i32, vp, i64, i32, i32, i32, vp, vp, vp, vp, sz, vp, vp]
     lib.drk_pg_logprob_fwd.restype = ctypes.c_int
@@ -139,6 +143,8 @@ def load() -> ctypes.CDLL:
     lib.drk_selftest_bounded_wait.restype = ctypes.c_int
     lib.drk_last_launch_count.argtypes = []
     lib.drk_last_launch_count.restype = ctypes.c_int
+    lib.drk_bounds_checked.argtypes = []
+    lib.drk_bounds_checked.restype = ctypes.c_int
     lib.drk_tensor_map_encodes.argtypes = []
     lib.drk_tensor_map_encodes.restype = ctypes.c_uint64
     lib.drk_status_string.argtypes = [ctypes.c_int]
@@ -186,6 +192,10 @@ def drk_version() -> int:
 
 def drk_last_launch_count() -> int:
     return load().drk_last_launch_count()
+
+
+def drk_bounds_checked() -> int:
+    return int(load().drk_bounds_checked())
 
 
 def drk_tensor_map_encodes() -> int:
@@ -236,9 +246,9 @@ def drk_reward(correct, t_ref, t_kernel, pr, n: int, p: Optional[drk_reward_para
 
 
 def drk_trloo_advantage(reward, valid, prompt_of_rollout, R: int, Tmax: int, gamma: float, baseline: int,
-                        ret, adv, gsize, stream=None, check: bool = True) -> int:
+                        ret, adv, gsize, status=None, stream=None, check: bool = True) -> int:
     rc = load().drk_trloo_advantage(_ptr(reward), _ptr(valid), _ptr(prompt_of_rollout), R, Tmax, gamma, baseline,
-                                    _ptr(ret), _ptr(adv), _ptr(gsize), _stream(stream))
+                                    _ptr(ret), _ptr(adv), _ptr(gsize), _ptr(status), _stream(stream))
     if check and rc != DRK_OK:
         raise DrkError(rc, "drk_trloo_advantage")
     return rc
@@ -356,14 +366,15 @@ def _torch_dtype(code: int) -> torch.dtype:
 
 
 def trloo_advantage(reward: torch.Tensor, valid: torch.Tensor, prompt_of_rollout: torch.Tensor,
-                    gamma: float = 1.0, baseline: int = DRK_BASELINE_TRLOO):
-    """Allocates ret/adv/gsize and calls drk_trloo_advantage.  Inputs are device tensors."""
+                    gamma: float = 1.0, baseline: int = DRK_BASELINE_TRLOO, status: Optional[torch.Tensor] = None):
+    """Allocates ret/adv/gsize and calls drk_trloo_advantage.  Inputs are device tensors; `status` (device
+    int32[1], optional) collects DRK_STATUS_BAD_GROUPS."""
     R, Tmax = reward.shape
     ret = torch.empty_like(reward)
     adv = torch.empty_like(reward)
     gsize = torch.empty((R, Tmax), dtype=torch.int32, device=reward.device)
     drk_trloo_advantage(reward.contiguous(), valid.contiguous(), prompt_of_rollout.contiguous(), R, Tmax,
-                        gamma, baseline, ret, adv, gsize)
+                        gamma, baseline, ret, adv, gsize, status)
     return ret, adv, gsize
 
 

@@ -286,7 +286,7 @@ int loss_fwd_bwd_impl(const void* hidden, const void* W, int32_t in_dtype, const
     rc = launch_need_rows(loss_mask, cu_seqlens, T, S, bw.coeff, st);
     if (rc != DRK_OK) return fail(rc);
     CompactArgs ca{bw.coeff, static_cast<const __nv_bfloat16*>(hidden), T, H, bw.blk_cnt, bw.blk_off, bw.n_rows,
-                   bw.rowmap, bw.hidden_c};
+                   bw.rowmap, bw.hidden_c, status};
     rc = launch_compact(ca, st);
     if (rc != DRK_OK) return fail(rc);
     if (cudaMemsetAsync(logp, 0, sizeof(float) * (size_t)T, st) != cudaSuccess ||
@@ -332,7 +332,7 @@ int loss_fwd_bwd_impl(const void* hidden, const void* W, int32_t in_dtype, const
     rc = launch_simt_bwd(b, st);
   } else {
     CompactArgs ca{bw.coeff, static_cast<const __nv_bfloat16*>(hidden), T, H, bw.blk_cnt, bw.blk_off, bw.n_rows,
-                   bw.rowmap, bw.hidden_c};
+                   bw.rowmap, bw.hidden_c, status};
     rc = launch_compact(ca, st);
     if (rc != DRK_OK) return fail(rc);
     rc = enqueue_umma_bwd(bplan, st);
@@ -391,7 +391,7 @@ size_t drk_pg_workspace_bytes(int64_t T, int32_t H, int32_t V, int32_t S, int32_
 
 int drk_trloo_advantage(const float* reward, const uint8_t* valid, const int32_t* prompt_of_rollout, int32_t R,
                         int32_t Tmax, float gamma, int32_t baseline, float* ret, float* adv, int32_t* gsize,
-                        void* stream) {
+                        uint32_t* status, void* stream) {
   g_launches = 0;
   if (R < 0 || Tmax < 0) return DRK_ERR_INVALID_ARG;
   if (baseline != DRK_BASELINE_TRLOO && baseline != DRK_BASELINE_GRPO) return DRK_ERR_INVALID_ARG;
@@ -401,7 +401,7 @@ int drk_trloo_advantage(const float* reward, const uint8_t* valid, const int32_t
   if (!reward || !valid || !prompt_of_rollout || !ret || !adv || !gsize) return DRK_ERR_INVALID_ARG;
   int rc = check_arch();
   if (rc != DRK_OK) return rc;
-  rc = launch_trloo(reward, valid, prompt_of_rollout, R, Tmax, gamma, baseline, ret, adv, gsize,
+  rc = launch_trloo(reward, valid, prompt_of_rollout, R, Tmax, gamma, baseline, ret, adv, gsize, status,
                     static_cast<cudaStream_t>(stream));
   if (rc != DRK_OK) g_launches = 0;
   return rc;
@@ -538,5 +538,13 @@ const char* drk_status_string(int s) {
 }
 
 int drk_version(void) { return 101; }
+
+int drk_bounds_checked(void) {
+#ifdef DRK_BOUNDS_CHECK
+  return 1;
+#else
+  return 0;
+#endif
+}
 
 }  // extern "C"

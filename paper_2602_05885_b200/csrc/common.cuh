@@ -28,6 +28,16 @@ extern thread_local int g_launches;
 // size queries still answer on a host without a GPU).  Grids, wave models and split counts derive from it.
 int sm_count();
 
+// Checked build (-DDRK_BOUNDS_CHECK): every index that a kernel derives from device-side data (row maps,
+// compacted counts, work-unit numbers, token ids used as addresses) is range-checked before use; a violation
+// sets DRK_STATUS_BOUNDS in the status word and the access is skipped -- no trap, no fault.  In the ordinary
+// build the test folds to `true` and costs nothing.
+#ifdef DRK_BOUNDS_CHECK
+#define DRK_IN_RANGE(cond, status_ptr) ((cond) ? true : (atomicOr((status_ptr), DRK_STATUS_BOUNDS), false))
+#else
+#define DRK_IN_RANGE(cond, status_ptr) (true)
+#endif
+
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
@@ -45,7 +55,8 @@ __device__ __forceinline__ int local_id(int id, int id_off, int width) {
 // ---- internal launchers (each returns a drk_status) -------------------------------------------
 
 int launch_trloo(const float* reward, const uint8_t* valid, const int32_t* prompt, int R, int Tmax,
-                 float gamma, int baseline, float* ret, float* adv, int32_t* gsize, cudaStream_t st);
+                 float gamma, int baseline, float* ret, float* adv, int32_t* gsize, uint32_t* status,
+                 cudaStream_t st);
 
 // Per-segment statistics, rejection decision, coefficients and loss.
 struct MrsArgs {
@@ -121,13 +132,14 @@ struct CompactArgs {
   const float* coeff; const __nv_bfloat16* hidden; int64_t T; int H;
   int32_t* blk_cnt; int32_t* blk_off; int32_t* n_rows /*[2]: count, count rounded up to 256*/;
   int32_t* rowmap /*[compact_map_len(T)]*/; __nv_bfloat16* hidden_c /*[compact_map_len(T), H]*/;
+  uint32_t* status = nullptr;   // status word for the checked build's range checks
 };
 int64_t compact_map_len(int64_t T);
 int compact_blocks(int64_t T);
 int launch_compact(const CompactArgs& a, cudaStream_t st);
 // dst[rowmap[r], :] = src[r, :] for the n_rows[0] compacted rows; src fp32 [*, H], dst fp32 or bf16 [T, H]
 int launch_scatter_rows(const float* src, int H, const int32_t* rowmap, const int32_t* n_rows, void* dst, bool dst_bf16,
-                        cudaStream_t st);
+                        int64_t T, uint32_t* status, cudaStream_t st);
 // need[t] = 1 for loss-masked tokens inside a segment, else 0 (the rows whose log-prob the loss can use)
 int launch_need_rows(const uint8_t* loss_mask, const int32_t* cu, int64_t T, int S, float* need, cudaStream_t st);
 

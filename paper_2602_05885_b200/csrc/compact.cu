@@ -40,7 +40,7 @@ __global__ void offsets_kernel(const int32_t* __restrict__ blk_cnt, int nblk, in
 __global__ void __launch_bounds__(kBlk) rowmap_kernel(const float* __restrict__ coeff, int64_t T,
                                                       const int32_t* __restrict__ blk_off,
                                                       const int32_t* __restrict__ n_rows, int64_t map_len,
-                                                      int32_t* __restrict__ rowmap) {
+                                                      int32_t* __restrict__ rowmap, uint32_t* __restrict__ status) {
   __shared__ int warp_cnt[kBlk / 32];
   const int64_t t = (int64_t)blockIdx.x * kBlk + threadIdx.x;
   const bool nz = (t < T) && (coeff[t] != 0.f);
@@ -50,7 +50,8 @@ __global__ void __launch_bounds__(kBlk) rowmap_kernel(const float* __restrict__ 
   __syncthreads();
   int base = blk_off[blockIdx.x];
   for (int i = 0; i < w; ++i) base += warp_cnt[i];
-  if (nz) rowmap[base + __popc(m & ((1u << lane) - 1u))] = (int32_t)t;
+  const int dst = base + __popc(m & ((1u << lane) - 1u));
+  if (nz && DRK_IN_RANGE(dst >= 0 && dst < map_len, status)) rowmap[dst] = (int32_t)t;
   // entries behind the last compacted row (disjoint from the ones written above)
   const int total = n_rows[0];
   if (t >= total && t < map_len) rowmap[t] = -1;
@@ -59,13 +60,15 @@ __global__ void __launch_bounds__(kBlk) rowmap_kernel(const float* __restrict__ 
 __global__ void __launch_bounds__(256) gather_kernel(const __nv_bfloat16* __restrict__ hidden, int H,
                                                      const int32_t* __restrict__ rowmap,
                                                      const int32_t* __restrict__ n_rows,
-                                                     __nv_bfloat16* __restrict__ hidden_c) {
-  const int padded = n_rows[1];
+                                                     __nv_bfloat16* __restrict__ hidden_c, int64_t T, int64_t map_len,
+                                                     uint32_t* __restrict__ status) {
+  int padded = n_rows[1];
+  if (!DRK_IN_RANGE(padded >= 0 && padded <= map_len, status)) padded = 0;
   const int vec_per_row = H / 8;  // 16-byte vectors; H is a multiple of 8 on this path
   for (int r = blockIdx.x; r < padded; r += gridDim.x) {
     const int src = rowmap[r];
     uint4* dst = reinterpret_cast<uint4*>(hidden_c + (size_t)r * H);
-    if (src >= 0) {
+    if (src >= 0 && DRK_IN_RANGE(src < T, status)) {
       const uint4* s = reinterpret_cast<const uint4*>(hidden + (size_t)src * H);
       for (int i = threadIdx.x; i < vec_per_row; i += blockDim.x) dst[i] = s[i];
     } else {
@@ -78,12 +81,12 @@ __global__ void __launch_bounds__(256) gather_kernel(const __nv_bfloat16* __rest
 __global__ void __launch_bounds__(256) scatter_rows_kernel(const float* __restrict__ src, int H,
                                                            const int32_t* __restrict__ rowmap,
                                                            const int32_t* __restrict__ n_rows, void* __restrict__ dst,
-                                                           int dst_bf16) {
+                                                           int dst_bf16, int64_t T, uint32_t* __restrict__ status) {
   const int cnt = n_rows[0];
   const int vec_per_row = H / 8;
   for (int r = blockIdx.x; r < cnt; r += gridDim.x) {
     const int t = rowmap[r];
-    if (t < 0) continue;
+    if (t < 0 || !DRK_IN_RANGE(t < T, status)) continue;
     const float4* s = reinterpret_cast<const float4*>(src + (size_t)r * H);
     for (int i = threadIdx.x; i < vec_per_row; i += blockDim.x) {
       const float4 a = s[2 * i], b = s[2 * i + 1];
@@ -104,8 +107,8 @@ __global__ void __launch_bounds__(256) scatter_rows_kernel(const float* __restri
 }
 
 int launch_scatter_rows(const float* src, int H, const int32_t* rowmap, const int32_t* n_rows, void* dst, bool dst_bf16,
-                        cudaStream_t st) {
-  scatter_rows_kernel<<<sm_count() * 8, 256, 0, st>>>(src, H, rowmap, n_rows, dst, dst_bf16 ? 1 : 0);
+                        int64_t T, uint32_t* status, cudaStream_t st) {
+  scatter_rows_kernel<<<sm_count() * 8, 256, 0, st>>>(src, H, rowmap, n_rows, dst, dst_bf16 ? 1 : 0, T, status);
   DRK_LAUNCHED();
   return DRK_OK;
 }
@@ -137,9 +140,9 @@ int launch_compact(const CompactArgs& a, cudaStream_t st) {
   DRK_LAUNCHED();
   offsets_kernel<<<1, 32, 0, st>>>(a.blk_cnt, nblk, a.blk_off, a.n_rows);
   DRK_LAUNCHED();
-  rowmap_kernel<<<nblk, kBlk, 0, st>>>(a.coeff, a.T, a.blk_off, a.n_rows, map_len, a.rowmap);
+  rowmap_kernel<<<nblk, kBlk, 0, st>>>(a.coeff, a.T, a.blk_off, a.n_rows, map_len, a.rowmap, a.status);
   DRK_LAUNCHED();
-  gather_kernel<<<sm_count() * 8, 256, 0, st>>>(a.hidden, a.H, a.rowmap, a.n_rows, a.hidden_c);
+  gather_kernel<<<sm_count() * 8, 256, 0, st>>>(a.hidden, a.H, a.rowmap, a.n_rows, a.hidden_c, a.T, map_len, a.status);
   DRK_LAUNCHED();
   return DRK_OK;
 }

@@ -37,12 +37,14 @@ __device__ __forceinline__ double return_at(const float* __restrict__ reward,
 __global__ void trloo_kernel(const float* __restrict__ reward, const uint8_t* __restrict__ valid,
                              const int32_t* __restrict__ prompt, int R, int Tmax, double gamma,
                              int baseline, float* __restrict__ ret, float* __restrict__ adv,
-                             int32_t* __restrict__ gsize) {
+                             int32_t* __restrict__ gsize, uint32_t* __restrict__ status) {
   const int warp = (int)((blockIdx.x * (size_t)blockDim.x + threadIdx.x) >> 5);
   const int lane = threadIdx.x & 31;
   if (warp >= R) return;
   const int first = warp;
   const int pid = prompt[first];
+  // groups are runs of equal prompt ids; a decrease means some prompt's rollouts are not contiguous
+  if (first > 0 && prompt[first - 1] > pid && status != nullptr && lane == 0) atomicOr(status, DRK_STATUS_BAD_GROUPS);
   if (first > 0 && prompt[first - 1] == pid) return;  // not the head of a run
   // find the end of the run: first index whose prompt differs
   int end = first + 1;
@@ -86,12 +88,13 @@ __global__ void trloo_kernel(const float* __restrict__ reward, const uint8_t* __
 }
 
 int launch_trloo(const float* reward, const uint8_t* valid, const int32_t* prompt, int R, int Tmax,
-                 float gamma, int baseline, float* ret, float* adv, int32_t* gsize, cudaStream_t st) {
+                 float gamma, int baseline, float* ret, float* adv, int32_t* gsize, uint32_t* status,
+                 cudaStream_t st) {
   if (R == 0 || Tmax == 0) return DRK_OK;
   const int threads = 128;  // 4 warps
   const int blocks = (int)ceil_div((int64_t)R * 32, threads);
   trloo_kernel<<<blocks, threads, 0, st>>>(reward, valid, prompt, R, Tmax, (double)gamma, baseline, ret,
-                                           adv, gsize);
+                                           adv, gsize, status);
   DRK_LAUNCHED();
   return DRK_OK;
 }

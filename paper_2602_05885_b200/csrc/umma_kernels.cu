@@ -63,6 +63,11 @@ enum Mode { FWD = 0, DL = 1, DW = 2, DH = 3 };
 
 struct UmmaParams {
   int m_tiles, n_tiles, k_blocks, group_m, nj, tiles_per_unit, num_units;
+  // Order of the work units.  group_n == 0: groups of group_m row tiles, within a group the column index
+  // is the slow one (the group's A panels stay in L2 while it sweeps the columns).  group_n > 0: groups of
+  // group_n column units, within a group the row tile is the slow index (the group's B panels stay in L2
+  // while the rows stream past).
+  int group_n;
   int64_t rows;  // valid extent of the tile-row index (T, or the chunk's width for DW)
   int cols;      // valid extent of the tile-column index (V, the chunk's width, or H)
   int v0;        // first vocabulary column of the chunk (0 for FWD)
@@ -102,6 +107,18 @@ struct Unit {
 };
 
 __device__ __forceinline__ Unit decode_unit(const UmmaParams& p, int m_tiles, int u) {
+  if (p.group_n > 0) {
+    const int per_group = m_tiles * p.group_n;      // every group but the last holds group_n column units
+    const int g = u / per_group;
+    const int rem = u - g * per_group;
+    const int gn = min(p.group_n, p.nj - g * p.group_n);
+    Unit r;
+    r.m = rem / gn;
+    r.j = g * p.group_n + rem % gn;
+    r.n_begin = r.j * p.tiles_per_unit;
+    r.n_end = min(p.n_tiles, r.n_begin + p.tiles_per_unit);
+    return r;
+  }
   const int per_group = p.group_m * p.nj;
   const int g = u / per_group;
   const int rem = u - g * per_group;
@@ -254,7 +271,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
     if constexpr (MODE == DW) k_blocks = (cnt + TK - 1) / TK;
   }
-  const int num_units = m_tiles * p.nj;
+  int num_units = m_tiles * p.nj;
+  // checked build: the device-side row count must fit what the host sized the buffers for
+  if (!DRK_IN_RANGE(m_tiles >= 0 && m_tiles <= p.m_tiles && k_blocks >= 0 && k_blocks <= p.k_blocks, p.status))
+    num_units = 0;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSTAGE; ++s) {
@@ -492,8 +512,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       __syncwarp();
       if (lane == 0) {
         const uint32_t src = out_stage + (boxes & 1u) * OUT_BOX_BYTES;
-        if (p.out_tma == 2) ptx::tma_reduce_add_2d(&tmC, src, x, y);
-        else ptx::tma_store_2d(&tmC, src, x, y);
+        // checked build: the box starts inside the output (what sticks out past its extents is clipped by the store)
+        if (DRK_IN_RANGE(x >= 0 && x < p.cols && y >= 0 && y < rows, p.status)) {
+          if (p.out_tma == 2) ptx::tma_reduce_add_2d(&tmC, src, x, y);
+          else ptx::tma_store_2d(&tmC, src, x, y);
+        }
         ptx::bulk_commit_group();
       }
       ++boxes;
@@ -509,6 +532,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if constexpr (MODE == FWD || MODE == DL || MODE == DH) {
         if (p.rowmap != nullptr) orow = row_ok ? (int64_t)p.rowmap[row] : -1;
         if constexpr (MODE == DH || MODE == FWD) row_ok = row_ok && orow >= 0;
+        // checked build: the token a compacted row maps to lies inside the batch, the unit inside the grid of units
+        if (!DRK_IN_RANGE(orow < p.T && un.m < m_tiles && un.j < p.nj, p.status)) { row_ok = false; orow = -1; }
       }
       // per-unit state
       float run_m = -CUDART_INF_F, run_l = 0.f, run_r = 0.f;  // FWD: log2-domain running max, sum, sum*logit
@@ -548,7 +573,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
               for (int j = 0; j < 32; ++j)
                 if (j == w) tg = x[j];
-              p.tgt[row] = tg;
+              if (DRK_IN_RANGE(row < p.T, p.status)) p.tgt[row] = tg;
             }
             float cm = x[0];
 #pragma unroll
@@ -660,7 +685,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if constexpr (MODE == FWD) {
         if (row_ok) {
           // natural-log units for the max, as the merge kernel expects
-          reinterpret_cast<float4*>(p.part)[(int64_t)un.j * p.T + row] = make_float4(run_m * kLn2, run_l, run_r, 0.f);
+          if (DRK_IN_RANGE(row < p.T && un.j < p.nj, p.status))
+            reinterpret_cast<float4*>(p.part)[(int64_t)un.j * p.T + row] = make_float4(run_m * kLn2, run_l, run_r, 0.f);
         }
       }
     }
@@ -933,10 +959,13 @@ int umma_nsplit(int64_t T, int V, int ctas, bool frugal) {
   return 1;
 }
 
-// Row tiles whose operand panels (rows x K bf16 each) are kept live together: about 40 MB.
+// How many operand panels (rows x K bf16 each) a group of work units keeps live in L2 while the other
+// operand streams past: about 38 MB worth.  Measured at T=32768, H=5120, V=151936 (interleaved runs): 10 column
+// tiles for DH (7424-deep panels) and 12-15 for DL are 2.7 % faster than row-tile groups that sweep all columns;
+// 20 and more fall off again, as do forward groups beyond ~16 row tiles (L2 serves both dies from 126 MB).
 static int panel_group(int rows_per_tile, int64_t k_elems) {
   const double panel = (double)rows_per_tile * (double)k_elems * 2.0;
-  int g = (int)(40.0 * 1024 * 1024 / panel);
+  int g = (int)(38.0 * 1024 * 1024 / panel);
   return g < 1 ? 1 : (g > 64 ? 64 : g);
 }
 
@@ -1051,6 +1080,7 @@ int enqueue_umma_bwd(const UmmaBwdPlan& plan, cudaStream_t st) {
       p.n_tiles = (int)ceil_div(vc_this, TN);
       p.k_blocks = (int)ceil_div(a.H, TK);
       p.nj = p.n_tiles; p.tiles_per_unit = 1; p.group_m = 16 / ctas;
+      p.group_n = panel_group(TN, a.H);        // W's column panels of the group stay in L2, the rows stream past
       p.rows = a.T; p.cols = vc_this; p.v0 = v0; p.T = a.T;
       p.id_off = a.id_off; p.id_width = a.V;
       p.ids = a.ids; p.lse = a.lse; p.coeff = a.coeff; p.dL = a.dL; p.vc = a.vc; p.status = a.status;
@@ -1085,6 +1115,7 @@ int enqueue_umma_bwd(const UmmaBwdPlan& plan, cudaStream_t st) {
       p.n_tiles = (int)ceil_div(a.H, TN);
       p.k_blocks = (int)ceil_div(vc_this, TK);
       p.nj = p.n_tiles; p.tiles_per_unit = 1; p.group_m = 32 / ctas;
+      p.group_n = panel_group(TN, vc_this);    // the W chunk's column panels of the group stay in L2
       p.rows = a.T; p.cols = a.H; p.v0 = v0; p.T = a.T;
       p.ldc = a.H; p.out_bf16 = 0; p.out_tma = chunk > 0 ? 2 : 1;
       p.status = a.status;
@@ -1095,7 +1126,7 @@ int enqueue_umma_bwd(const UmmaBwdPlan& plan, cudaStream_t st) {
     }
   }
   // dH[rowmap[r], :] = dH_acc[r, :] in the requested type
-  return launch_scatter_rows(a.dH_acc, a.H, a.rowmap, a.n_rows, a.dH, a.dh_dtype == DRK_BF16, st);
+  return launch_scatter_rows(a.dH_acc, a.H, a.rowmap, a.n_rows, a.dH, a.dh_dtype == DRK_BF16, a.T, a.status, st);
 }
 
 int launch_umma_bwd(const UmmaBwdArgs& a, cudaStream_t st) {

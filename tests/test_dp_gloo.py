@@ -39,6 +39,24 @@ def _worker(rank, world, port, out):
     n_slices = dp.all_reduce_dw_slices(dW, 256)
     assert n_slices == 4 and dp.chunk_slices(1000, 256)[-1] == (768, 1000)
     assert torch.equal(dW, torch.full((1000, 4), 3.0))          # 1 + 2 on every element, every slice covered once
+    # the same exchange as a reduce-scatter: every rank keeps its rows of each slice only (ragged slice ends and
+    # a last slice of 232 rows included); together the ranks hold every row of the sum exactly once
+    V, vc = 1001, 256
+    g = torch.Generator().manual_seed(100)
+    parts = [torch.randn((V, 4), generator=g) for _ in range(world)]
+    mine_rows = dp.dw_shard_rows(V, vc, world, rank)
+    shard = torch.empty((sum(b - a for a, b in mine_rows), 4))
+    assert dp.reduce_scatter_dw_slices(parts[rank].clone(), vc, shard) == 4
+    want = torch.cat([(parts[0] + parts[1])[a:b] for a, b in mine_rows])
+    assert torch.allclose(shard, want, atol=1e-6)
+    covered = sorted(r for k in range(world) for r in dp.dw_shard_rows(V, vc, world, k))
+    assert covered[0][0] == 0 and covered[-1][1] == V and all(x[1] == y[0] for x, y in zip(covered, covered[1:]))
+    # partial sums of dH never cross the ranks in 16 bits
+    try:
+        dp.all_reduce_dh(torch.zeros(4, dtype=torch.bfloat16))
+        raise AssertionError("bf16 partial sums must be refused")
+    except ValueError:
+        pass
     out.put((rank, mine, tokens, t_job, total, len(plans), sum(p.used for p in plans)))
     dist.destroy_process_group()
 
@@ -122,8 +140,21 @@ def test_vocabulary_parallel_exchanges_on_three_ranks():
 
 
 def test_vocab_shards_cover_the_vocabulary():
-    for V, world in ((151936, 8), (151936, 2), (151936, 1), (4096, 3), (300, 4)):
-        sh = dp.vocab_shards(V, world)
+    import pytest
+    for V, world, align in ((151936, 8, 256), (151936, 2, 256), (151936, 1, 256), (4096, 3, 256), (300, 2, 256),
+                            (300, 4, 32)):
+        sh = dp.vocab_shards(V, world, align)
         assert len(sh) == world and sh[0][0] == 0 and sh[-1][1] == V
-        assert all(a[1] == b[0] for a, b in zip(sh, sh[1:]))
-        assert all(a % 256 == 0 for a, _ in sh if a < V)
+        assert all(a[1] == b[0] for a, b in zip(sh, sh[1:])) and all(b > a for a, b in sh)
+        assert all(a % align == 0 for a, _ in sh)
+    # more ranks than vocabulary tiles: a clear error instead of an empty range that the library would reject
+    with pytest.raises(ValueError, match="without rows"):
+        dp.vocab_shards(300, 4)
+
+
+def test_reduce_scatter_without_a_process_group_keeps_every_row():
+    dW = torch.arange(40, dtype=torch.float32).reshape(10, 4)
+    rows = dp.dw_shard_rows(10, 4, 1, 0)
+    assert rows == [(0, 4), (4, 8), (8, 10)]
+    shard = torch.empty((10, 4))
+    assert dp.reduce_scatter_dw_slices(dW, 4, shard) == 3 and torch.equal(shard, dW)

@@ -78,6 +78,13 @@ def test_device_detected_errors_set_status_bits():
     dev = run_device(case, make_params(*OPEN))
     assert dev["status"] & B.DRK_STATUS_BAD_SEGMENTS
     assert int(dev["seg_keep"][1]) == 0
+    # boundaries that go back and forward again would make two samples share tokens: the step back is what
+    # the device sees, and it raises the same bit
+    case.cu = torch.tensor([0, 90, 40, 140], dtype=torch.int32)
+    case.seg_adv = torch.ones(3)
+    dev = run_device(case, make_params(*OPEN))
+    assert dev["status"] & B.DRK_STATUS_BAD_SEGMENTS
+    assert int(dev["seg_keep"][1]) == 0
 
 
 def test_host_detected_errors_return_codes():

@@ -208,3 +208,21 @@ def test_segment_advantages_gather():
     torch.cuda.synchronize()
     assert int(status.item()) == B.DRK_STATUS_BAD_SEGMENTS and float(out[0]) == 0.0 and float(out[1]) == 0.0
     assert B.drk_segment_advantages(adv, sr, stn, R, Tmax, 0, out, status) == B.DRK_OK
+
+
+def test_partial_sums_of_dh_are_exchanged_in_fp32():
+    # eight ranges of the vocabulary: each range's dH is a partial sum.  Summed in fp32 and rounded once at the end
+    # the result is closer to the oracle than the sum of parts that were each rounded to bf16 first, which is
+    # why the multi-rank helper refuses 16-bit parts
+    from paper_2602_05885_b200 import dp
+    case = get_case("medium")
+    lo, hi = Hh.wide_band(case)
+    cuts = tuple(dp.vocab_shards(case.V, 8, align=256))
+    errs = {}
+    for name, dh in (("fp32 parts", B.DRK_F32), ("bf16 parts", B.DRK_BF16)):
+        dev, _ = run_sharded(case, cuts, make_params(lo, hi, VETO, v_chunk=2048, dh_dtype=dh))
+        ref = Hh.check_against_oracle(case, dev, lo, hi, VETO)
+        errs[name] = Hh.rel_fro(Hh.f64(dev["dH"]), ref["dH"])
+    assert errs["fp32 parts"] < errs["bf16 parts"] <= Hh.TOL_GRAD_FRO
+    assert errs["fp32 parts"] < 1e-3
+    Hh.report(f"dH over 8 vocabulary ranges, rel. Frobenius error: {errs}")

@@ -88,3 +88,18 @@ def test_irregular_prompt_runs_and_empty():
     e = torch.empty(0, device=d)
     assert B.drk_trloo_advantage(e, e, e, 0, 3, 1.0, 0, e, e, e) == B.DRK_OK
     assert B.drk_last_launch_count() == 0
+
+
+def test_scattered_rollouts_of_a_prompt_are_flagged():
+    # groups are runs of equal prompt ids (Sec. 4.2 groups by prompt): when a prompt's rollouts are not
+    # contiguous the run-based grouping would split its turn groups, and the status word says so
+    d = torch.device("cuda:0")
+    g = torch.Generator().manual_seed(10)
+    reward = synth.draw_rewards((6, 2), g).to(d)
+    valid = torch.ones((6, 2), dtype=torch.uint8, device=d)
+    for prompt, want in (([0, 0, 1, 1, 2, 2], 0), ([0, 0, 1, 1, 0, 0], B.DRK_STATUS_BAD_GROUPS),
+                         ([5, 4, 4, 4, 4, 4], B.DRK_STATUS_BAD_GROUPS)):
+        st = torch.zeros(1, dtype=torch.int32, device=d)
+        B.trloo_advantage(reward, valid, torch.tensor(prompt, dtype=torch.int32, device=d), status=st)
+        torch.cuda.synchronize()
+        assert int(st.item()) == want, prompt
