@@ -533,7 +533,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (p.rowmap != nullptr) orow = row_ok ? (int64_t)p.rowmap[row] : -1;
         if constexpr (MODE == DH || MODE == FWD) row_ok = row_ok && orow >= 0;
         // checked build: the token a compacted row maps to lies inside the batch, the unit inside the grid of units
-        if (!DRK_IN_RANGE(orow < p.T && un.m < m_tiles && un.j < p.nj, p.status)) { row_ok = false; orow = -1; }
+        if (!DRK_IN_RANGE((p.rowmap == nullptr || orow < p.T) && un.m < m_tiles && un.j < p.nj, p.status)) {
+          row_ok = false;
+          orow = -1;
+        }
       }
       // per-unit state
       float run_m = -CUDART_INF_F, run_l = 0.f, run_r = 0.f;  // FWD: log2-domain running max, sum, sum*logit
