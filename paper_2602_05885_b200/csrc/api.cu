@@ -56,14 +56,20 @@ bool sizes_ok(int64_t T, int H, int V, int in_dtype) {
 // Chunk width for the tensor-core backward when the caller leaves it to the library: the multiple of
 // 256 that minimises the modelled time of the three per-chunk kernels.  Each kernel is persistent
 // over the device's SMs with 128x256 tiles, so its time is (waves of tiles) x (k-blocks per tile); a fixed
-// cost per launch stands for fill and drain.  The dL buffer is kept below ~512 MiB (or 8192 columns).
+// cost per launch stands for fill and drain, and each chunk costs one more pass over the fp32 dH accumulator
+// (T x H elements read and written through the memory-side add).  The dL buffer is kept below 2 GiB (a fifth of
+// the bf16 logits at T=32768, V=151936): measured there, 30720-column chunks (5 chunks) are 2.5 % faster than
+// 7424-column ones (21 chunks), 14848 (11 chunks) 1.2 %; callers short of memory pass a smaller v_chunk.
 int auto_vchunk(int64_t T, int H, int V) {
   const int64_t sms = sm_count(), launch_cost = 96;
   const int64_t mt_T = ceil_div(T, 128), nt_H = ceil_div(H, 256), kb_H = ceil_div(H, 64), kb_T = ceil_div(T, 64);
-  int64_t cap = ((int64_t)1 << 29) / (2 * (T > 0 ? T : 1)) / 256 * 256;
+  int64_t cap = ((int64_t)1 << 31) / (2 * (T > 0 ? T : 1)) / 256 * 256;
   if (cap < 8192) cap = 8192;
   if (cap > 32768) cap = 32768;
   const int64_t vmax = ceil_div(V, 256) * 256;
+  // one accumulate pass over dH, in the model's unit (a 128x256x64 MMA block): T*H*8 bytes of traffic at about
+  // the rate at which such a block's operands (48 KiB) stream in
+  const double acc_pass = (double)T * (double)H * 8.0 / (48.0 * 1024.0) / (double)sms;
   int best = 0;
   double best_cost = 0;
   for (int64_t vc = 2048; vc <= cap; vc += 256) {
@@ -73,6 +79,7 @@ int auto_vchunk(int64_t T, int H, int V) {
       cost += (double)(ceil_div(mt_T * ceil_div(w, 256), sms) * kb_H + launch_cost);   // DL
       cost += (double)(ceil_div(ceil_div(w, 128) * nt_H, sms) * kb_T + launch_cost);   // DW
       cost += (double)(ceil_div(mt_T * nt_H, sms) * ceil_div(w, 64) + launch_cost);    // DH
+      cost += acc_pass;
     }
     if (best == 0 || cost < best_cost) { best = (int)vc; best_cost = cost; }
     if (vc >= vmax) break;

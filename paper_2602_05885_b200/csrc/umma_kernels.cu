@@ -1118,7 +1118,10 @@ int enqueue_umma_bwd(const UmmaBwdPlan& plan, cudaStream_t st) {
       p.n_tiles = (int)ceil_div(a.H, TN);
       p.k_blocks = (int)ceil_div(vc_this, TK);
       p.nj = p.n_tiles; p.tiles_per_unit = 1; p.group_m = 32 / ctas;
-      p.group_n = panel_group(TN, vc_this);    // the W chunk's column panels of the group stay in L2
+      // the W chunk's column panels of the group stay in L2 where they fit; with deep chunks (long panels) at
+      // least ten column tiles per group keep the set of tiles in flight about square (rows x columns)
+      p.group_n = panel_group(TN, vc_this);
+      if (p.group_n < 10) p.group_n = 10;
       p.rows = a.T; p.cols = a.H; p.v0 = v0; p.T = a.T;
       p.ldc = a.H; p.out_bf16 = 0; p.out_tma = chunk > 0 ? 2 : 1;
       p.status = a.status;
