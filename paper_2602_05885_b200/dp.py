@@ -179,7 +179,7 @@ def all_reduce_dh(dH_part: torch.Tensor) -> torch.Tensor:
 
 
 def vocab_parallel_loss_fwd_bwd(hidden, W_shard, ids, rollout_logp, loss_mask, cu_seqlens, seg_adv, v_begin: int,
-                                V_total: int, p, bufs, stats=None, stream=None):
+                                V_total: int, p, bufs, stats=None, stream=None, dh_out=None):
     """One fused loss step with W split by rows over the process group: statistics of this rank's rows,
     all-gather, loss and this rank's gradient parts, all-reduce of dH.  `bufs` is a PgLossBuffers built for
     V = W_shard.shape[0]; on return bufs.dW holds this rank's rows of dW and bufs.dH the complete dH.
