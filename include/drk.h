@@ -373,6 +373,14 @@ int drk_last_launch_count(void);
  */
 uint64_t drk_tensor_map_encodes(void);
 
+/*
+ * Host-side fault injection for tests of the error contract (no counterpart in the paper): the nth next request
+ * for a tensor map inside this process fails as if the driver had refused to encode it (nth >= 1; 0 clears a
+ * pending injection).  The call that hits it returns DRK_ERR_CUDA, and because all maps are built before the
+ * first enqueue it must leave the stream and every output untouched.  Nothing on the device is made to fail.
+ */
+void drk_selftest_fail_tensor_map(int32_t nth);
+
 const char* drk_status_string(int status);
 int drk_version(void);
 /* 1 if this library was compiled with -DDRK_BOUNDS_CHECK (see DRK_STATUS_BOUNDS), else 0. */

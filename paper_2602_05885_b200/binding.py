@@ -143,6 +143,8 @@ def load() -> ctypes.CDLL:
     lib.drk_selftest_bounded_wait.restype = ctypes.c_int
     lib.drk_last_launch_count.argtypes = []
     lib.drk_last_launch_count.restype = ctypes.c_int
+    lib.drk_selftest_fail_tensor_map.argtypes = [i32]
+    lib.drk_selftest_fail_tensor_map.restype = None
     lib.drk_bounds_checked.argtypes = []
     lib.drk_bounds_checked.restype = ctypes.c_int
     lib.drk_tensor_map_encodes.argtypes = []
@@ -192,6 +194,10 @@ def drk_version() -> int:
 
 def drk_last_launch_count() -> int:
     return load().drk_last_launch_count()
+
+
+def drk_selftest_fail_tensor_map(nth: int) -> None:
+    load().drk_selftest_fail_tensor_map(int(nth))
 
 
 def drk_bounds_checked() -> int:

@@ -532,6 +532,8 @@ int drk_last_launch_count(void) { return g_launches; }
 
 uint64_t drk_tensor_map_encodes(void) { return umma_map_encodes(); }
 
+void drk_selftest_fail_tensor_map(int32_t nth) { umma_fail_map_request(nth); }
+
 const char* drk_status_string(int s) {
   switch (s) {
     case DRK_OK: return "ok";

@@ -788,6 +788,9 @@ std::unordered_map<MapKey, CUtensorMap, MapKeyHash>& map_table() {
   return *t;
 }
 std::atomic<uint64_t> g_map_encodes{0};
+// Host-side fault injection for tests: when positive, the n-th next request for a tensor map fails as if the
+// driver had refused to encode it (cached or not).
+std::atomic<int> g_fail_map_in{0};
 
 // Row-major matrix [outer, inner] of 2-byte (bf16) or 4-byte (fp32) elements with row pitch `pitch_elems`;
 // box = box_inner x box_outer, 128-byte swizzle, zero fill outside the extents on loads (stores are clipped).
@@ -795,6 +798,7 @@ bool make_map_typed(CUtensorMap* m, const void* base, uint64_t inner, uint64_t o
                     uint32_t box_inner, uint32_t box_outer, bool f32) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
+  if (g_fail_map_in.load(std::memory_order_relaxed) > 0 && g_fail_map_in.fetch_sub(1) == 1) return false;
   const uint32_t esz = f32 ? 4 : 2;
   const MapKey key{base, inner, outer, pitch_elems * esz, box_inner, box_outer, f32 ? 1u : 0u};
   {
@@ -922,6 +926,7 @@ int launch_mode(int ctas, const CUtensorMap& a, const CUtensorMap& b, const CUte
 }  // namespace
 
 uint64_t umma_map_encodes() { return g_map_encodes.load(std::memory_order_relaxed); }
+void umma_fail_map_request(int nth) { g_fail_map_in.store(nth > 0 ? nth : 0); }
 
 // Number of vocabulary ranges per row tile in the forward (each work unit = one row tile x one range,
 // with its own partial max / sum-exp per row).

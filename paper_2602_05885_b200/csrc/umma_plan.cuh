@@ -29,5 +29,7 @@ int enqueue_umma_bwd(const UmmaBwdPlan& plan, cudaStream_t st);
 
 // Tensor maps encoded so far by this process (cache misses); steady-state calls add none.
 uint64_t umma_map_encodes();
+// Test hook: the nth next tensor-map request fails (0 clears a pending injection).
+void umma_fail_map_request(int nth);
 
 }  // namespace drk

@@ -225,3 +225,35 @@ def test_steady_state_calls_encode_no_tensor_maps(engine):
     B.pg_loss_fwd_bwd(*ins, p, bufs2)
     torch.cuda.synchronize()
     assert torch.equal(bufs2.dW, first[1]) and torch.equal(bufs2.dH, first[2])
+
+
+def test_a_failing_host_step_enqueues_nothing():
+    # every tensor map of the forward and of all chunks of the backward is built before the first enqueue: when
+    # the k-th request fails (injected on the host), the call reports DRK_ERR_CUDA and neither the outputs nor
+    # the status word nor the stream have been touched, whichever map it was
+    d = torch.device("cuda:0")
+    case = Hh.build_plain_case("inject", T=300, H=128, V=1500, dtype=torch.bfloat16, S=3, seed=32)
+    p = make_params(*OPEN, v_chunk=512)          # three chunks: 2 forward maps + 4 + 3 * 4 + 1 backward maps
+    ins = [t.to(d) for t in (case.hidden, case.W, case.ids, case.rollout_logp, case.loss_mask, case.cu, case.seg_adv)]
+    code = B.DRK_BF16
+    for nth in (1, 2, 3, 7, 12, 19):
+        bufs = B.PgLossBuffers(case.T, case.H, case.V, case.S, code, p, d)
+        for t in (bufs.logp, bufs.lse, bufs.dH, bufs.dW, bufs.loss):
+            t.fill_(float("nan"))
+        torch.cuda.synchronize()
+        B.drk_selftest_fail_tensor_map(nth)
+        rc = B.drk_pg_loss_fwd_bwd(ins[0], ins[1], code, ins[2], ins[3], ins[4], ins[5], ins[6], case.T, case.H, case.V,
+                                   case.S, p, bufs.loss, bufs.logp, bufs.lse, bufs.entropy, bufs.seg_w, bufs.seg_keep,
+                                   bufs.counters, bufs.dH, bufs.dW, bufs.workspace, bufs.workspace_bytes, bufs.status,
+                                   check=False)
+        B.drk_selftest_fail_tensor_map(0)
+        torch.cuda.synchronize()
+        assert rc == B.DRK_ERR_CUDA, nth
+        assert B.drk_last_launch_count() == 0
+        assert int(bufs.status.item()) == 0
+        for t in (bufs.logp, bufs.lse, bufs.dH, bufs.dW, bufs.loss):
+            assert torch.isnan(t.float()).all(), nth
+    # and the next ordinary call is unaffected
+    dev = run_device(case, p)
+    assert dev["status"] == 0
+    Hh.check_against_oracle(case, dev, *OPEN)
