@@ -161,7 +161,10 @@ typedef struct {
   int32_t dw_accumulate; /* 0: dW = gradient; 1: dW += gradient (accumulation over micro-batches)    */
   int32_t engine;        /* drk_engine; default DRK_ENGINE_AUTO                                      */
   int32_t v_chunk;       /* vocabulary columns whose dLogits are held at once in the backward;
-                            0 = library default; rounded up to a multiple of 256                    */
+                            0 = library default (a bf16 buffer of at most 2 GiB: 31232 columns at
+                            T = 32768; wider chunks mean fewer passes over the dH accumulator, a
+                            smaller value trades a few percent of speed for workspace); rounded up
+                            to a multiple of 256                                                    */
   int32_t keep_from_caller; /* 0: seg_keep is an output, decided by MRS here.  1: seg_keep is an INPUT:
                             the caller has already decided which samples are retained (e.g. a sample
                             split over several micro-batches, judged on log-probs from

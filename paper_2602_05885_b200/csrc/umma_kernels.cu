@@ -2,20 +2,22 @@
 //
 // One persistent, warp-specialised GEMM kernel, instantiated for the four contractions of the path:
 //
-//   FWD : S = hidden W^T tile by tile; epilogue keeps a running (max, sum-exp) per row over the
-//         unit's vocabulary range and picks out the sampled token's logit.  Logits never leave
-//         the SM.
-//   DL  : the same tiles for one vocabulary chunk; epilogue stores
+//   FWD : S = hidden W^T tile by tile; epilogue keeps a running (max, sum-exp, sum-exp*logit) per row over
+//         the unit's vocabulary range and picks out the sampled token's logit.  Logits never leave the SM.
+//   DL  : the same tiles for one vocabulary chunk; epilogue forms
 //         dL = c_t (exp(s - lse_t) - onehot) as bf16 into the chunk buffer [T, vc].
 //   DW  : dW[chunk] (+)= dL^T hidden        (both operands have M/N contiguous: MN-major)
-//   DH  : dH (+)= dL W[chunk]               (A K-major, B MN-major)
+//   DH  : dH_acc (+)= dL W[chunk]           (A K-major, B MN-major; fp32 accumulator over the compacted rows)
 //
-// Tile 128 x 256 x 64, one CTA per SM, 192 threads:
-//   warp 0    : TMA producer (one lane): 128B-swizzled operand tiles into a ring of stages
-//   warp 1    : tensor-memory allocation; one lane issues tcgen05.mma (4 per stage, K = 16 each)
-//               into one of two 256-column fp32 accumulators and commits to mbarriers
+// Tile 128 x 256 x 64 per CTA (256 x 256 per CTA pair with cta_group::2), one CTA per SM, 192 threads:
+//   warp 0    : TMA producer (one lane): 128B-swizzled operand tiles into a ring of stages; in the even
+//               CTA it also draws the block's next work unit from a device-side counter and announces it
+//   warp 1    : tensor-memory allocation; one lane issues tcgen05.mma (K = 16 each) into one of two
+//               256-column fp32 accumulators and commits to mbarriers
 //   warps 2-5 : epilogue; warp w reads tensor-memory lanes 32*(w%4)..+31, one accumulator row per
-//               thread, 32 columns per tcgen05.ld, while the MMA warp fills the other accumulator
+//               thread, 32 columns per tcgen05.ld, while the MMA warp fills the other accumulator.
+//               DL / DW / DH stage their output in swizzled shared memory and let the TMA unit store it
+//               (or add it, at the memory side, to what is there).
 // Every mbarrier wait is bounded; on expiry the block raises DRK_STATUS_TIMEOUT, drains its
 // in-flight copies and MMAs, frees tensor memory and returns.
 #include "common.cuh"
@@ -930,10 +932,10 @@ void umma_fail_map_request(int nth) { g_fail_map_in.store(nth > 0 ? nth : 0); }
 
 // Number of vocabulary ranges per row tile in the forward (each work unit = one row tile x one range,
 // with its own partial max / sum-exp per row).
-//  - default: ranges of two 256-column tiles.  Short units, taken in an order that keeps ~40 MB of hidden
+//  - default: ranges of two 256-column tiles.  Short units, taken in an order that keeps ~38 MB of hidden
 //    panels (a group of row tiles) live while the group sweeps the vocabulary, let L2 serve most operand
-//    re-reads: measured at T=32768, H=5120, V=151936 the forward drops from ~44 to ~38.5 ms and its DRAM
-//    reads from ~130 GB to 40-70 GB against four long ranges per row tile.
+//    re-reads: measured at T=32768, H=5120, V=151936 the forward dropped from ~44 to ~38.5 ms against four
+//    long ranges per row tile, and to 35.5 ms (16 GB of DRAM reads) once the units were drawn dynamically.
 //  - frugal: the fewest ranges that fill whole waves (within 1 % of the best wave efficiency), for
 //    callers with little scratch for the partials.
 int umma_nsplit(int64_t T, int V, int ctas, bool frugal) {
