@@ -314,7 +314,8 @@ int drk_pg_loss_fwd_bwd(const void* hidden, const void* W, int32_t in_dtype, con
  *          entropy, seg_w, seg_keep and counters come out identical on every rank;
  *          dW_shard [V_local, H] = rows v_begin.. of dW, final;
  *          dH_part [T, H] = sum over the rank's columns of dL[t,v] W[v,:]
- *   4. all-reduce (sum) of dH_part over the ranks = dH.  p->dh_dtype = DRK_F32 keeps that sum in fp32.
+ *   4. all-reduce (sum) of dH_part over the ranks = dH.  With more than one rank set p->dh_dtype = DRK_F32 and
+ *      convert after the reduction: a part rounded to bf16 first loses bits that the sum would have kept.
  *
  * ids hold token numbers of the whole vocabulary, 0 <= ids[t] < V_total; ids outside set DRK_STATUS_BAD_ID in
  * step 3.  Workspace: drk_pg_workspace_bytes(T, H, V_local, S, in_dtype, p, which) with which = 0 for step 1
