@@ -53,3 +53,50 @@ def test_dense_operands_and_draws():
                                  cu_seqlens=cu)
     assert (noise[:500].abs() < 1.0).all() and (noise[500:].abs() >= 2.0).sum() >= 3
     assert u.min() >= 0 and u.max() < 1
+
+
+def test_threshold_between_never_sits_on_a_value():
+    import random
+    rnd = random.Random(3)
+    for n in (2, 3, 5, 6, 16, 19, 28, 33):
+        vals = [rnd.random() for _ in range(n)]
+        q = synth.threshold_between(vals)
+        assert all(abs(q - v) > 0 for v in vals)
+        below = sum(v < q for v in vals)
+        assert 0 < below < n and abs(below - n / 2) <= max(1.5, 0.2 * n)      # about half on either side
+        gaps = sorted(vals)
+        lo = max(v for v in vals if v < q)
+        hi = min(v for v in vals if v > q)
+        assert abs(q - 0.5 * (lo + hi)) < 1e-15                                # midway between its neighbours
+    assert synth.threshold_between([]) > 0 and synth.threshold_between([0.25]) == 0.5
+
+
+def test_nudged_samples_land_inside_the_paper_band_with_margin():
+    # the input recipe of the parity tests: a seeded 15 % of the clean samples get a mean log-ratio inside
+    # +-6e-4, at least 4e-4 away from the edges ln 0.999 / ln 1.001; samples with outlier tokens are left alone
+    import math
+    import numpy as np
+    from tests import helpers as Hh
+    rng = np.random.default_rng(0)
+    S, L = 20, 200
+    cu = np.arange(0, (S + 1) * L, L)
+    T = S * L
+    logp = -rng.random(T) * 8
+    noise = rng.normal(0, 0.1, T)
+    noise[3 * L + 5] = -9.5                    # an outlier token in sample 3
+    mask = (rng.random(T) < 0.9).astype(np.uint8)
+    rl = (logp + noise).astype(np.float32)
+    out = Hh.nudge_into_band(logp, rl, mask, cu, seed=1)
+    assert out.dtype == np.float32
+    moved = []
+    for g in range(S):
+        sel = mask[cu[g]:cu[g + 1]].astype(bool)
+        before = (logp[cu[g]:cu[g + 1]] - rl[cu[g]:cu[g + 1]].astype(np.float64))[sel].mean()
+        after = (logp[cu[g]:cu[g + 1]] - out[cu[g]:cu[g + 1]].astype(np.float64))[sel].mean()
+        if abs(before - after) > 1e-9:
+            moved.append(g)
+            assert abs(after) <= 6e-4 + 1e-6
+            assert min(abs(after - math.log(0.999)), abs(after - math.log(1.001))) >= 3.9e-4
+            # unmasked tokens are untouched
+            assert np.array_equal(out[cu[g]:cu[g + 1]][~sel], rl[cu[g]:cu[g + 1]][~sel])
+    assert len(moved) == max(2, round(0.15 * 19)) and 3 not in moved
