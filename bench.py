@@ -263,6 +263,9 @@ def main():
     ap.add_argument("--v-chunk", type=int, default=0)
     ap.add_argument("--forward-rows", default="all", choices=["all", "usable"],
                     help="usable: the forward skips rows that are not loss-masked tokens of a segment")
+    ap.add_argument("--dw-exchange", default="all-reduce", choices=["all-reduce", "reduce-scatter"],
+                    help="with --sync-dw: all-reduce every finished slice of dW, or reduce-scatter it so that each rank "
+                         "keeps its 1/N of the rows (half the bytes; what a sharded optimizer needs)")
     ap.add_argument("--sync-dw", action="store_true",
                     help="all-reduce dW across ranks slice by slice as the backward finishes each vocabulary chunk "
                          "(overlapped on a second stream); off by default: the loss path itself needs no collective")
@@ -359,6 +362,10 @@ def main():
             e.record(stream)
         B.set_dw_chunk_events(p, [e.cuda_event for e in events])
         comm = torch.cuda.Stream()
+        dw_shard = None
+        if args.dw_exchange == "reduce-scatter":
+            owned = dp.dw_shard_rows(V, vc, world, rank)
+            dw_shard = torch.empty((sum(b - a for a, b in owned), H), dtype=bufs.dW.dtype, device=dev)
 
     def step(hidden, ids, rl, mask, cu, out=None):
         o = out if out is not None else bufs
@@ -376,8 +383,11 @@ def main():
                               o.workspace, o.workspace_bytes, o.status, stream)
         launches[0] += B.drk_last_launch_count()
         if comm is not None:
-            dp.all_reduce_dw_slices(bufs.dW, vc, events, comm)
-            stream.wait_stream(comm)        # the step ends when the last slice has been reduced
+            if dw_shard is not None:
+                dp.reduce_scatter_dw_slices(bufs.dW, vc, dw_shard, events, comm)
+            else:
+                dp.all_reduce_dw_slices(bufs.dW, vc, events, comm)
+            stream.wait_stream(comm)        # the step ends when the last slice has been exchanged
 
     def barrier():
         if world > 1:
@@ -560,7 +570,7 @@ def main():
                        "parallelism": (f"vp{world}: W split by rows ({V} of {V_total} on rank 0), one micro-batch for "
                                        "all ranks; all-gather of per-row statistics, all-reduce of dH") if vocab else
                                       (f"dp{world}: one micro-batch per rank, " +
-                                       ("dW all-reduced per vocabulary chunk, overlapped" if args.sync_dw
+                                       (f"dW exchanged per vocabulary chunk ({args.dw_exchange}), overlapped" if args.sync_dw
                                         else "no collective on the loss path"))},
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s",
                          "frac": achieved / peaks["tflops"], "traffic": traffic, "traffic_source": traffic_note,
